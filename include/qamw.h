@@ -1,0 +1,181 @@
+/*
+ * qamw.h -- C ABI of the QAM-W weight codec for NVIDIA B200 (sm_100a).
+ *
+ * The codec quantises a weight matrix W[d_out, d_in] row by row (paper, Section 3):
+ *   encode:  x = W D_s (Section B.2)  ->  r = |x|_2, u = x / r (Section 3.1 step 1)
+ *            ->  y = F S u, sign-masked block-Hadamard rotation (step 2, Lemma 1)
+ *            ->  pairs z_k = (y_2k, y_2k+1) / sigma_k (steps 3-4, Section 3.4)
+ *            ->  idx_k = nearest entry of one 2-D codebook (step 5, Section 3.6)
+ *            ->  B = log2 K bits per pair, bit-packed (step 6)
+ *   decode:  unpack -> codeword -> x sigma_k -> S F -> x r -> / s_j -> bf16 (Section 3.2, B.2)
+ *
+ * General rules
+ *   - Every function returns QAMW_OK (0) or a negative QAMW_ERR_* code; nothing throws, aborts,
+ *     prints or traps.  Argument errors are detected on the host before anything is launched.
+ *   - "device" pointers are CUDA global-memory addresses on the current device, "host" pointers
+ *     are ordinary process memory.  The caller owns every buffer; the library allocates device
+ *     memory only inside a qamw_codebook (released by qamw_codebook_destroy).
+ *   - Device-side functions are asynchronous: they enqueue kernels on `stream` (a cudaStream_t
+ *     passed as void*, NULL = the default stream) and return without synchronising.
+ *   - Matrices are row-major.  W is f32 or bf16 (QAMW_DTYPE_*), with `w_row_stride` elements
+ *     between rows; every row must start on a 16-byte boundary.
+ *   - Packed rows start `packed_row_stride` bytes apart (>= qamw_packed_row_bytes, a multiple
+ *     of 4); index k of a row occupies stream bits [k*B, (k+1)*B), stream bit t being bit
+ *     (t mod 8) of byte floor(t/8); padding bits up to the row stride are written as zero.
+ *   - Arithmetic contract of the encoder (what makes indices reproducible bit for bit):
+ *       t_j = f32(s_j) * sign_j;  x_j = f32(f32(W_ij) * t_j);
+ *       r_i = f32(sqrt(sum_j (double)x_j^2));
+ *       h   = f32 butterfly of x per block, stages 1, 2, 4, ..., b/2, (a, b) -> (a+b, a-b);
+ *       y_j = f32(h_j * g),  g = f32(1 / ((double)r_i * sqrt((double)b)));
+ *       z   = f32(y * q_k),  q_k = f32(1 / (double)sigma_k);
+ *       idx = argmin_c fma(dy, dy, dx*dx) in f32 with dx = z_x - c_x, dy = z_y - c_y,
+ *             lowest index among equal distances.
+ *     A row with r_i == 0 is encoded as the origin's codeword in every pair and decodes to zeros.
+ *     A row whose norm is not finite sets bit 0 of *status_out; its indices are unspecified.
+ */
+#ifndef QAMW_H_
+#define QAMW_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QAMW_OK 0
+#define QAMW_ERR_ARG (-1)       /* NULL pointer, value out of range */
+#define QAMW_ERR_SHAPE (-2)     /* d_in odd, block does not divide d_in, K / block not a power of two */
+#define QAMW_ERR_ALIGN (-3)     /* pointer or stride alignment */
+#define QAMW_ERR_CUDA (-4)      /* a CUDA runtime call failed */
+#define QAMW_ERR_NONFINITE (-5) /* reported by qamw_status_to_error for a non-finite row norm */
+#define QAMW_ERR_NOMEM (-6)     /* workspace too small / shared memory budget exceeded */
+
+#define QAMW_DTYPE_F32 0
+#define QAMW_DTYPE_BF16 1
+
+#define QAMW_FLAG_BRUTE_FORCE 1u /* encode: exhaustive search over all K instead of the cell table */
+
+#define QAMW_DEFAULT_SIGN_SEED 0x51A5C0DEC0FFEE01ULL
+#define QAMW_MAX_BLOCK 1024 /* cap of Section 3.3 */
+#define QAMW_MAX_K 4096
+#define QAMW_CALIB_MAX_ROWS 1024 /* "up to 1024 unit-normalized rows" (Section 3.4) */
+
+typedef struct {
+    int32_t d_out, d_in;       /* d_in even, block | d_in */
+    int32_t block;             /* b = 2^q, 2 <= b <= 1024 */
+    int32_t K;                 /* codebook size, power of two, 2 <= K <= 4096 */
+    int32_t w_dtype;           /* QAMW_DTYPE_* of W */
+    uint32_t flags;            /* QAMW_FLAG_* */
+    int64_t w_row_stride;      /* elements between rows of W (>= d_in) */
+    int64_t packed_row_stride; /* bytes between packed rows */
+} qamw_params;
+
+typedef struct qamw_codebook qamw_codebook; /* opaque: device copy of C plus its exact search table */
+
+/* ----------------------------------------------------------------------------------------------
+ * Host-side helpers (host pointers only, no CUDA calls).
+ * -------------------------------------------------------------------------------------------- */
+
+/* Section 3.6: "trained by Lloyd iterations on the unit circular Gaussian".  Sample-based Lloyd
+ * on n_samples Box-Muller samples of counter stream `seed` (u = ((mix64(mix64(seed ^
+ * 0xD1B54A32D192ED03) + golden*(n+1)) >> 11) + 0.5) * 2^-53, sample i from counters 2i, 2i+1);
+ * initial codewords sqrt(2) * sample_i; each iteration assigns every sample to its nearest
+ * codeword and moves each codeword to the mean of its cell (empty cells stay); stops when the
+ * training MSE improves by no more than rel_tol (relative) or after max_iters updates; the result
+ * is sorted by (squared radius, angle) and rounded to f32.
+ * codebook_out: host, K*2 floats (x, y interleaved).  train_mse_out: host, may be NULL; receives
+ * the mean squared distance of the samples to the returned f32 codebook. */
+int qamw_train_codebook(int K, uint64_t n_samples, uint64_t seed, int max_iters, double rel_tol,
+                        float* codebook_out, double* train_mse_out);
+
+/* Section B.2: s_j = clamp(r_j^alpha / geomean(r^alpha), 1/16, 16); r_j floored at FLT_MIN;
+ * alpha == 0 gives all ones.  act_rms, s_out: host, d_in floats. */
+int qamw_channel_scales(const float* act_rms, int d_in, float alpha, float* s_out);
+
+/* Sign mask of Appendix A.1 ("deterministic sequence generated from a fixed 64-bit seed"):
+ * sign_j = -1 if the top bit of mix64(seed + 0x9E3779B97F4A7C15*(j+1)) is set, else +1, with
+ * mix64 the SplitMix64 finaliser.  signs_out: host, d_in bytes of +1 / -1. */
+int qamw_make_signs(uint64_t seed, int d_in, int8_t* signs_out);
+
+/* Section 3.3: largest power of two dividing d_in, capped at 1024 (2048 -> 1024, 5632 -> 512).
+ * Returns 0 for d_in <= 0. */
+int qamw_block_size_rule(int d_in);
+
+/* Section 3.1 step 6: ceil((d_in/2) * log2(K) / 8); 0 on invalid arguments. */
+size_t qamw_packed_row_bytes(int d_in, int K);
+
+/* Section 3.7 equation: log2(K)/2 + 16/d_in, plus 16/d_out when channel scales are stored. */
+double qamw_bpw(int d_out, int d_in, int K, int has_channel_scales);
+
+/* Maps the status word written by qamw_encode / qamw_calibrate to QAMW_OK or QAMW_ERR_NONFINITE. */
+int qamw_status_to_error(int32_t status_word);
+
+/* ----------------------------------------------------------------------------------------------
+ * Codebook object.
+ * -------------------------------------------------------------------------------------------- */
+
+/* Uploads the K x 2 f32 codebook (host pointer) to the current device and builds the exact
+ * spatial search table used by qamw_encode: a uniform grid over the codebook's bounding square
+ * whose every cell lists all codewords whose nearest-neighbour region can meet the cell, so that
+ * the table search returns the same index as an exhaustive search (points outside the grid are
+ * searched exhaustively).  Synchronous.  *out must be released with qamw_codebook_destroy. */
+int qamw_codebook_create(const float* codebook_host, int K, qamw_codebook** out);
+void qamw_codebook_destroy(qamw_codebook* cb);
+
+/* Introspection for tests and benchmarks (host values): grid side, number of candidate entries,
+ * largest candidate list, bytes of shared memory the table occupies. */
+int qamw_codebook_table_info(const qamw_codebook* cb, int32_t* grid_out, int32_t* n_candidates_out,
+                             int32_t* max_list_out, int32_t* table_bytes_out);
+
+/* ----------------------------------------------------------------------------------------------
+ * Device-side entry points.  chan_scale (d_in floats) may be NULL = no channel scaling;
+ * signs: d_in bytes of +1/-1; sigma: d_in/2 floats; all device pointers.
+ * -------------------------------------------------------------------------------------------- */
+
+/* Bytes of device scratch qamw_calibrate needs for these parameters. */
+size_t qamw_calibrate_workspace_bytes(const qamw_params* p);
+
+/* Section 3.4 equation: sigma_k = mean_i |(y_2k, y_2k+1)| / sqrt(pi/2) over n = min(d_out, 1024)
+ * rows i = floor(t*d_out/n), rows of zero norm skipped, y as in the arithmetic contract above;
+ * floored at 1e-4/sqrt(d_in); 1/sqrt(d_in) when no row qualifies.  The column means are
+ * accumulated in double, per thread block and then in a fixed order, so the result is
+ * reproducible.  workspace: device scratch of at least qamw_calibrate_workspace_bytes(p) bytes,
+ * 8-byte aligned, overwritten.  status_out: device int32, bit 0 set if a row norm was not finite
+ * (may be NULL). */
+int qamw_calibrate(const void* W, const qamw_params* p, const float* chan_scale, const int8_t* signs,
+                   float* sigma_out, void* workspace, size_t workspace_bytes, int32_t* status_out,
+                   void* stream);
+
+/* Section 3.1 steps 1-6 (after Section B.2 scaling) for all rows.  Writes packed_out
+ * [d_out, packed_row_stride] bytes, row_norm_out [d_out] f32 and ORs bit 0 into *status_out
+ * (device int32, caller-zeroed, may be NULL) for non-finite rows. */
+int qamw_encode(const void* W, const qamw_params* p, const float* chan_scale, const int8_t* signs,
+                const float* sigma, const qamw_codebook* cb, uint8_t* packed_out, float* row_norm_out,
+                int32_t* status_out, void* stream);
+
+/* Diagnostic variant of the encoder front half: writes y (the rotated unit direction, before the
+ * division by sigma) as f32 [d_out, d_in] and the row norms; used to check stage-wise parity. */
+int qamw_rotate(const void* W, const qamw_params* p, const float* chan_scale, const int8_t* signs,
+                float* y_out, float* row_norm_out, int32_t* status_out, void* stream);
+
+/* Section 3.2 + B.2: W_hat[d_out, d_in] bf16 (row stride d_in) from the packed stream. */
+int qamw_decode(const uint8_t* packed, const float* row_norm, const float* chan_scale,
+                const int8_t* signs, const float* sigma, const qamw_codebook* cb, const qamw_params* p,
+                void* w_hat_bf16_out, void* stream);
+
+/* Corollary 3 / Corollary 4 sums in double:
+ *   out4[0] = sum (W - W_hat)^2        out4[1] = sum W^2
+ *   out4[2] = sum r_j^2 (W - W_hat)^2  out4[3] = sum r_j^2 W^2     (r_j = act_rms, 1 if NULL)
+ * so that rho_w = sqrt(out4[0]/out4[1]) and the diagonal-M_x rho_o = sqrt(out4[2]/out4[3]).
+ * W as described by p; W_hat bf16 with row stride d_in; out4: device, 4 doubles, overwritten. */
+int qamw_distortion(const void* W, const void* w_hat_bf16, const float* act_rms, const qamw_params* p,
+                    double* out4, void* stream);
+
+/* Last CUDA error string seen by the library on this thread (host, static storage). */
+const char* qamw_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QAMW_H_ */
