@@ -116,17 +116,27 @@ int qamw_status_to_error(int32_t status_word);
  * -------------------------------------------------------------------------------------------- */
 
 /* Uploads the K x 2 f32 codebook (host pointer) to the current device and builds the exact
- * spatial search table used by qamw_encode: a uniform grid over the codebook's bounding square
- * whose every cell lists all codewords whose nearest-neighbour region can meet the cell, so that
- * the table search returns the same index as an exhaustive search (points outside the grid are
- * searched exhaustively).  Synchronous.  *out must be released with qamw_codebook_destroy. */
-int qamw_codebook_create(const float* codebook_host, int K, qamw_codebook** out);
+ * spatial search table used by qamw_encode (Section 3.6: "nearest codebook entry by Euclidean
+ * distance"): [-8, 8)^2 is cut into grid x grid cells whose boundaries follow the quantiles of
+ * N(0, 2); every cell lists all codewords whose nearest-neighbour region can meet the cell, so a
+ * scan of the list returns what a scan of the whole codebook returns.  Points outside [-8, 8)^2
+ * are scanned exhaustively.  grid = 0 picks a default (about 2.1 sqrt(K)).  Synchronous.
+ * *out must be released with qamw_codebook_destroy on the same device. */
+int qamw_codebook_create(const float* codebook_host, int K, int grid, qamw_codebook** out);
 void qamw_codebook_destroy(qamw_codebook* cb);
 
-/* Introspection for tests and benchmarks (host values): grid side, number of candidate entries,
- * largest candidate list, bytes of shared memory the table occupies. */
-int qamw_codebook_table_info(const qamw_codebook* cb, int32_t* grid_out, int32_t* n_candidates_out,
-                             int32_t* max_list_out, int32_t* table_bytes_out);
+/* Introspection (host values): info_out[0..5] = grid side, total candidate entries, longest
+ * candidate list, number of cells with more than four candidates, overflow entries, table bytes. */
+int qamw_codebook_table_info(const qamw_codebook* cb, int32_t* info_out);
+
+/* Host-only construction of the same table, for inspection and tests (no CUDA).  lut_out: 4096
+ * bytes mapping fine bin floor(z*256 + 2048) to a grid column/row; cells_out: grid*grid records of
+ * four u16 (ascending candidate indices, last repeated as padding; or {0xFFFF, offset, count, 0}
+ * pointing into overflow_out).  Any output pointer may be NULL; info_out as above (6 values).
+ * Returns QAMW_ERR_NOMEM if the table does not fit budget_bytes or a capacity. */
+int qamw_search_table_build(const float* codebook_host, int K, int grid, size_t budget_bytes,
+                            uint8_t* lut_out, uint16_t* cells_out, size_t cells_cap,
+                            uint16_t* overflow_out, size_t overflow_cap, int32_t* info_out);
 
 /* ----------------------------------------------------------------------------------------------
  * Device-side entry points.  chan_scale (d_in floats) may be NULL = no channel scaling;

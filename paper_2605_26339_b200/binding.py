@@ -1,0 +1,264 @@
+"""Thin ctypes binding of libqamw.so (same names as the C ABI in include/qamw.h).
+
+Only argument marshalling happens here: torch supplies device memory and the
+stream, every step of the codec runs inside the library's CUDA kernels.  There
+is no fallback: if the shared library is missing or a call fails, an exception
+is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+QAMW_OK = 0
+ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_CUDA, ERR_NONFINITE, ERR_NOMEM = -1, -2, -3, -4, -5, -6
+DTYPE_F32, DTYPE_BF16 = 0, 1
+FLAG_BRUTE_FORCE = 1
+DEFAULT_SIGN_SEED = 0x51A5C0DEC0FFEE01
+_ERR_NAMES = {-1: "QAMW_ERR_ARG", -2: "QAMW_ERR_SHAPE", -3: "QAMW_ERR_ALIGN", -4: "QAMW_ERR_CUDA",
+              -5: "QAMW_ERR_NONFINITE", -6: "QAMW_ERR_NOMEM"}
+
+EXPORTED = [
+    "qamw_train_codebook", "qamw_channel_scales", "qamw_make_signs", "qamw_block_size_rule",
+    "qamw_packed_row_bytes", "qamw_bpw", "qamw_status_to_error", "qamw_codebook_create",
+    "qamw_codebook_destroy", "qamw_codebook_table_info", "qamw_search_table_build",
+    "qamw_calibrate_workspace_bytes", "qamw_calibrate", "qamw_encode", "qamw_rotate", "qamw_decode",
+    "qamw_distortion", "qamw_last_cuda_error",
+]
+
+
+class QamwError(RuntimeError):
+    def __init__(self, fn: str, code: int, detail: str = ""):
+        self.code = code
+        super().__init__(f"{fn} failed: {_ERR_NAMES.get(code, code)} {detail}".strip())
+
+
+class Params(C.Structure):
+    _fields_ = [("d_out", C.c_int32), ("d_in", C.c_int32), ("block", C.c_int32), ("K", C.c_int32),
+                ("w_dtype", C.c_int32), ("flags", C.c_uint32), ("w_row_stride", C.c_int64),
+                ("packed_row_stride", C.c_int64)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libqamw.so from the package directory; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: run __graft_entry__.build() (nvcc, sm_100a) first; "
+                               "there is no CPU fallback")
+        L = C.CDLL(path)
+        vp, i32, u64, sz = C.c_void_p, C.c_int, C.c_uint64, C.c_size_t
+        L.qamw_train_codebook.argtypes = [i32, u64, u64, i32, C.c_double, vp, vp]
+        L.qamw_channel_scales.argtypes = [vp, i32, C.c_float, vp]
+        L.qamw_make_signs.argtypes = [u64, i32, vp]
+        L.qamw_block_size_rule.argtypes = [i32]
+        L.qamw_packed_row_bytes.argtypes = [i32, i32]
+        L.qamw_packed_row_bytes.restype = sz
+        L.qamw_bpw.argtypes = [i32, i32, i32, i32]
+        L.qamw_bpw.restype = C.c_double
+        L.qamw_status_to_error.argtypes = [C.c_int32]
+        L.qamw_codebook_create.argtypes = [vp, i32, i32, C.POINTER(vp)]
+        L.qamw_codebook_destroy.argtypes = [vp]
+        L.qamw_codebook_destroy.restype = None
+        L.qamw_codebook_table_info.argtypes = [vp, vp]
+        L.qamw_search_table_build.argtypes = [vp, i32, i32, sz, vp, vp, sz, vp, sz, vp]
+        L.qamw_calibrate_workspace_bytes.argtypes = [C.POINTER(Params)]
+        L.qamw_calibrate_workspace_bytes.restype = sz
+        L.qamw_calibrate.argtypes = [vp, C.POINTER(Params), vp, vp, vp, vp, sz, vp, vp]
+        L.qamw_encode.argtypes = [vp, C.POINTER(Params), vp, vp, vp, vp, vp, vp, vp, vp]
+        L.qamw_rotate.argtypes = [vp, C.POINTER(Params), vp, vp, vp, vp, vp, vp]
+        L.qamw_decode.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Params), vp, vp]
+        L.qamw_distortion.argtypes = [vp, vp, vp, C.POINTER(Params), vp, vp]
+        L.qamw_last_cuda_error.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def _check(fn: str, rc: int):
+    if rc != QAMW_OK:
+        detail = lib().qamw_last_cuda_error().decode() if rc == ERR_CUDA else ""
+        raise QamwError(fn, rc, detail)
+
+
+def _np(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _dp(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+# ------------------------------------------------------------------------------- host side
+def train_codebook(K: int, n_samples: int = 1 << 20, seed: int = 0, max_iters: int = 100,
+                   rel_tol: float = 1e-6) -> Tuple[np.ndarray, float]:
+    cb = np.empty((K, 2), np.float32)
+    mse = C.c_double()
+    _check("qamw_train_codebook", lib().qamw_train_codebook(K, n_samples, seed, max_iters, rel_tol,
+                                                           cb.ctypes.data, C.addressof(mse)))
+    return cb, mse.value
+
+
+def channel_scales(act_rms, alpha: float) -> np.ndarray:
+    r = _np(act_rms, np.float32)
+    out = np.empty_like(r)
+    _check("qamw_channel_scales", lib().qamw_channel_scales(r.ctypes.data, r.shape[0], alpha, out.ctypes.data))
+    return out
+
+
+def make_signs(seed: int, d_in: int) -> np.ndarray:
+    out = np.empty(d_in, np.int8)
+    _check("qamw_make_signs", lib().qamw_make_signs(seed, d_in, out.ctypes.data))
+    return out
+
+
+def block_size_rule(d_in: int) -> int:
+    return int(lib().qamw_block_size_rule(d_in))
+
+
+def packed_row_bytes(d_in: int, K: int) -> int:
+    return int(lib().qamw_packed_row_bytes(d_in, K))
+
+
+def bpw(d_out: int, d_in: int, K: int, has_channel_scales: bool) -> float:
+    return float(lib().qamw_bpw(d_out, d_in, K, int(has_channel_scales)))
+
+
+def status_to_error(status_word: int) -> int:
+    return int(lib().qamw_status_to_error(status_word))
+
+
+def search_table_build(codebook, grid: int = 0, budget_bytes: int = 1 << 20):
+    """Host-only table construction -> (lut u8[4096], cells u16[grid*grid,4], overflow u16[], info[6])."""
+    cb = _np(codebook, np.float32)
+    K = cb.shape[0]
+    info = np.zeros(6, np.int32)
+    _check("qamw_search_table_build", lib().qamw_search_table_build(cb.ctypes.data, K, grid, budget_bytes, None,
+                                                                    None, 0, None, 0, info.ctypes.data))
+    g = int(info[0])
+    lut = np.zeros(4096, np.uint8)
+    cells = np.zeros((g * g, 4), np.uint16)
+    ovf = np.zeros(max(1, int(info[4])), np.uint16)
+    _check("qamw_search_table_build", lib().qamw_search_table_build(cb.ctypes.data, K, g, budget_bytes,
+                                                                    lut.ctypes.data, cells.ctypes.data, cells.size,
+                                                                    ovf.ctypes.data, ovf.size, info.ctypes.data))
+    return lut, cells, ovf, info
+
+
+# ------------------------------------------------------------------------------- codebook object
+class Codebook:
+    """Owns a qamw_codebook* on the current CUDA device."""
+
+    def __init__(self, codebook, grid: int = 0):
+        cb = _np(codebook, np.float32)
+        if cb.ndim != 2 or cb.shape[1] != 2:
+            raise ValueError("codebook must be [K, 2]")
+        self.K = cb.shape[0]
+        self.host = cb.copy()
+        h = C.c_void_p()
+        _check("qamw_codebook_create", lib().qamw_codebook_create(cb.ctypes.data, self.K, grid, C.byref(h)))
+        self._h = h
+
+    @property
+    def handle(self):
+        return self._h
+
+    def table_info(self) -> np.ndarray:
+        info = np.zeros(6, np.int32)
+        _check("qamw_codebook_table_info", lib().qamw_codebook_table_info(self._h, info.ctypes.data))
+        return info
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().qamw_codebook_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+# ------------------------------------------------------------------------------- device side
+@dataclass
+class MatrixMeta:
+    """Device-resident per-matrix metadata shared by encode and decode."""
+    chan_scale: Optional[torch.Tensor]  # f32 [d_in] or None
+    signs: torch.Tensor  # int8 [d_in]
+    sigma: Optional[torch.Tensor]  # f32 [d_in/2]
+
+
+def make_params(W: Optional[torch.Tensor], d_out: int, d_in: int, block: int, K: int, flags: int = 0,
+                packed_row_stride: Optional[int] = None, w_dtype: Optional[int] = None) -> Params:
+    if W is not None:
+        if W.dtype == torch.float32:
+            w_dtype = DTYPE_F32
+        elif W.dtype == torch.bfloat16:
+            w_dtype = DTYPE_BF16
+        else:
+            raise TypeError("W must be float32 or bfloat16")
+        if W.dim() != 2 or W.stride(1) != 1:
+            raise ValueError("W must be 2-D with unit column stride")
+        stride = W.stride(0) if W.shape[0] > 1 else d_in
+    else:
+        stride = d_in
+        w_dtype = DTYPE_BF16 if w_dtype is None else w_dtype
+    if packed_row_stride is None:
+        packed_row_stride = default_packed_row_stride(d_in, K)
+    return Params(d_out, d_in, block, K, w_dtype, flags, stride, packed_row_stride)
+
+
+def default_packed_row_stride(d_in: int, K: int) -> int:
+    """Row payload rounded up to 4 bytes (16 when the payload already is a multiple of 16)."""
+    rb = packed_row_bytes(d_in, K)
+    return (rb + 3) // 4 * 4
+
+
+def calibrate_workspace_bytes(p: Params) -> int:
+    return int(lib().qamw_calibrate_workspace_bytes(C.byref(p)))
+
+
+def calibrate(W: torch.Tensor, p: Params, chan_scale, signs, sigma_out: torch.Tensor, workspace: torch.Tensor,
+              status: Optional[torch.Tensor] = None, stream=None):
+    _check("qamw_calibrate", lib().qamw_calibrate(_dp(W), C.byref(p), _dp(chan_scale), _dp(signs), _dp(sigma_out),
+                                                 _dp(workspace), workspace.numel() * workspace.element_size(),
+                                                 _dp(status), _stream(stream)))
+
+
+def encode(W: torch.Tensor, p: Params, chan_scale, signs, sigma, cb: Codebook, packed_out: torch.Tensor,
+           row_norm_out: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None):
+    _check("qamw_encode", lib().qamw_encode(_dp(W), C.byref(p), _dp(chan_scale), _dp(signs), _dp(sigma), cb.handle,
+                                           _dp(packed_out), _dp(row_norm_out), _dp(status), _stream(stream)))
+
+
+def rotate(W: torch.Tensor, p: Params, chan_scale, signs, y_out: torch.Tensor, row_norm_out: torch.Tensor,
+           status: Optional[torch.Tensor] = None, stream=None):
+    _check("qamw_rotate", lib().qamw_rotate(_dp(W), C.byref(p), _dp(chan_scale), _dp(signs), _dp(y_out),
+                                           _dp(row_norm_out), _dp(status), _stream(stream)))
+
+
+def decode(packed: torch.Tensor, row_norm: torch.Tensor, chan_scale, signs, sigma, cb: Codebook, p: Params,
+           w_hat_out: torch.Tensor, stream=None):
+    _check("qamw_decode", lib().qamw_decode(_dp(packed), _dp(row_norm), _dp(chan_scale), _dp(signs), _dp(sigma),
+                                           cb.handle, C.byref(p), _dp(w_hat_out), _stream(stream)))
+
+
+def distortion(W: torch.Tensor, w_hat: torch.Tensor, act_rms, p: Params, out4: torch.Tensor, stream=None):
+    _check("qamw_distortion", lib().qamw_distortion(_dp(W), _dp(w_hat), _dp(act_rms), C.byref(p), _dp(out4),
+                                                   _stream(stream)))

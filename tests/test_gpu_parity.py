@@ -1,0 +1,316 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.
+
+Exactness rules (from the benchmark spec of this codec):
+  * packed indices bit-exact, except pairs whose oracle best / second-best squared distances
+    differ by less than 1e-6 relative -- those are counted, and the GPU's choice must then be
+    one of the two near-tied codewords;
+  * rotated coordinates and row norms within 1e-5 relative (they are in fact required to be
+    bit-identical here, because the index rule needs identical 2-D points);
+  * decoded weights within 1 bf16 ulp given identical indices, plus the f32 butterfly's
+    absolute error bound 2^-21 * |block| for elements that nearly cancel;
+  * calibration within 1e-5 relative; distortion sums within 1e-9 relative.
+"""
+import numpy as np
+import pytest
+import torch
+
+from conftest import load_golden_codebook
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from paper_2605_26339_b200 import binding as q
+    from paper_2605_26339_b200 import synth
+
+DEV = "cuda:0"
+_codebooks = {}
+
+
+def _codebook(orc, K):
+    if K not in _codebooks:
+        if K >= 64:
+            host = load_golden_codebook(K)
+        else:  # tiny codebooks: trained by the oracle on the spot
+            host = orc.train_codebook(K, 1 << 12, 7, 30, 1e-6)[0]
+        _codebooks[K] = (host, q.Codebook(host))
+    return _codebooks[K]
+
+
+def _to_bits(W: torch.Tensor) -> np.ndarray:
+    if W.dtype == torch.bfloat16:
+        return W.cpu().view(torch.int16).numpy().view(np.uint16)
+    return W.cpu().numpy()
+
+
+def _make(d_out, d_in, dtype, seed, student=True):
+    g = torch.Generator().manual_seed(seed)
+    x = torch.randn((d_out, d_in), generator=g)
+    if student:
+        chi = sum(torch.randn((d_out, d_in), generator=g) ** 2 for _ in range(4)) / 4
+        x = x / chi.sqrt()
+    x = x * torch.exp(0.7 * torch.randn((d_out, 1), generator=g))
+    act = torch.exp(torch.randn(d_in, generator=g))
+    return x.to(dtype), act.numpy().astype(np.float32)
+
+
+def _bf16_ordered(bits: np.ndarray) -> np.ndarray:
+    b = bits.astype(np.int32)
+    return np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+
+
+class Case:
+    """Runs every GPU entry point on one matrix and keeps the outputs on the host."""
+
+    def __init__(self, orc, W: torch.Tensor, act, alpha, block, K, flags=0, row_sel=None, packed_stride=None):
+        self.orc, self.block, self.K = orc, block, K
+        d_out, d_in = W.shape
+        self.d_out, self.d_in = d_out, d_in
+        self.cb_host, self.cb = _codebook(orc, K)
+        self.s = q.channel_scales(act, alpha) if alpha else None
+        self.signs = q.make_signs(q.DEFAULT_SIGN_SEED, d_in)
+        Wd = W.to(DEV) if W.device.type == "cpu" else W
+        self.Wd = Wd
+        self.p = q.make_params(Wd, d_out, d_in, block, K, flags, packed_stride)
+        s_d = None if self.s is None else torch.from_numpy(self.s).to(DEV)
+        signs_d = torch.from_numpy(self.signs).to(DEV)
+        # rows the oracle looks at (all rows unless a sample is given)
+        self.rows = np.arange(d_out) if row_sel is None else np.asarray(row_sel)
+        self.W_rows = _to_bits(Wd[torch.from_numpy(self.rows).to(DEV)]) if row_sel is not None else _to_bits(Wd)
+
+        # calibration: GPU on the full matrix; oracle on the full matrix too (it reads <= 1024 rows)
+        ws = torch.empty(max(8, q.calibrate_workspace_bytes(self.p)), dtype=torch.uint8, device=DEV)
+        self.status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        sigma_d = torch.empty(d_in // 2, dtype=torch.float32, device=DEV)
+        q.calibrate(Wd, self.p, s_d, signs_d, sigma_d, ws, self.status)
+        self.sigma_gpu = sigma_d.cpu().numpy()
+        n_cal = min(d_out, 1024)
+        cal_rows = (np.arange(n_cal) * d_out) // n_cal
+        W_cal = _to_bits(Wd[torch.from_numpy(cal_rows).to(DEV)])
+        self.sigma, rc = orc.calibrate(W_cal, block, self.s, self.signs)
+        sigma_d = torch.from_numpy(self.sigma).to(DEV)  # both sides use the oracle's sigma from here on
+
+        self.y_d = torch.empty((d_out, d_in), dtype=torch.float32, device=DEV)
+        norm_rot = torch.empty(d_out, dtype=torch.float32, device=DEV)
+        q.rotate(Wd, self.p, s_d, signs_d, self.y_d, norm_rot, self.status)
+        self.norm_rot = norm_rot.cpu().numpy()
+
+        stride = self.p.packed_row_stride
+        packed_d = torch.full((d_out, stride), 0xAB, dtype=torch.uint8, device=DEV)
+        norm_d = torch.empty(d_out, dtype=torch.float32, device=DEV)
+        q.encode(Wd, self.p, s_d, signs_d, sigma_d, self.cb, packed_d, norm_d, self.status)
+        self.packed = packed_d.cpu().numpy()
+        self.norm = norm_d.cpu().numpy()
+
+        self.enc = orc.encode(self.W_rows, block, self.cb_host, self.s, self.signs, self.sigma,
+                              packed_row_stride=stride, diagnostics=True)
+        # decode the ORACLE's stream on the GPU ("given identical indices")
+        opacked = np.ascontiguousarray(self.enc["packed"])
+        pk = torch.from_numpy(opacked).to(DEV)
+        nm = torch.from_numpy(self.enc["row_norm"]).to(DEV)
+        what_d = torch.empty((len(self.rows), d_in), dtype=torch.bfloat16, device=DEV)
+        p_dec = q.make_params(None, len(self.rows), d_in, block, K, 0, stride)
+        q.decode(pk, nm, s_d, signs_d, sigma_d, self.cb, p_dec, what_d)
+        self.what = _to_bits(what_d)
+        # distortion of the GPU's own round trip on the full matrix
+        what_full = torch.empty((d_out, d_in), dtype=torch.bfloat16, device=DEV)
+        q.decode(packed_d, norm_d, s_d, signs_d, sigma_d, self.cb, self.p, what_full)
+        out4 = torch.empty(4, dtype=torch.float64, device=DEV)
+        act_d = torch.from_numpy(np.ascontiguousarray(act, np.float32)).to(DEV)
+        q.distortion(Wd, what_full, act_d, self.p, out4)
+        torch.cuda.synchronize()
+        self.out4 = out4.cpu().numpy()
+        self.what_full = _to_bits(what_full)
+        self.act = act
+        self.status_word = int(self.status.cpu()[0])
+
+    # ---- checks ------------------------------------------------------------------------------
+    def check_calibration(self):
+        np.testing.assert_allclose(self.sigma_gpu, self.sigma, rtol=1e-5)
+
+    def check_front_half(self):
+        y = self.y_d[torch.from_numpy(self.rows).to(DEV)].cpu().numpy()
+        zq = (1.0 / self.sigma.astype(np.float64)).astype(np.float32)
+        z_gpu = (y.reshape(len(self.rows), -1, 2) * zq[None, :, None]).astype(np.float32)
+        z_orc = self.enc["z"]
+        scale = np.abs(z_orc).max(axis=(1, 2), keepdims=True) + 1e-30
+        assert np.all(np.abs(z_gpu - z_orc) <= 1e-5 * scale)
+        np.testing.assert_allclose(self.norm[self.rows], self.enc["row_norm"], rtol=1e-5)
+        np.testing.assert_allclose(self.norm_rot[self.rows], self.enc["row_norm"], rtol=1e-5)
+        # value equality: -0.0 of an all-zero row counts as +0.0
+        same_z = np.array_equal(z_gpu, z_orc)
+        same_r = np.array_equal(self.norm[self.rows], self.enc["row_norm"])
+        return same_z, same_r
+
+    def check_indices(self):
+        B = int(np.log2(self.K))
+        n_pairs = self.d_in // 2
+        idx_gpu = np.stack([self.orc.unpack_row(self.packed[r], n_pairs, B) for r in self.rows])
+        idx_orc = self.enc["idx"]
+        d1, d2 = self.enc["d2_best"], self.enc["d2_second"]
+        diff = idx_gpu != idx_orc
+        exempt = (d2 - d1) < 1e-6 * d2
+        assert not np.any(diff & ~exempt), f"{int((diff & ~exempt).sum())} non-exempt index mismatches"
+        if diff.any():  # an exempt mismatch must still be one of the near-tied codewords
+            z = self.enc["z"].astype(np.float64)[diff]
+            c = self.cb_host[idx_gpu[diff]].astype(np.float64)
+            dg = ((z - c) ** 2).sum(1)
+            assert np.all(dg <= d2[diff] * (1 + 1e-9))
+        # padding up to the row stride is zero
+        rb = q.packed_row_bytes(self.d_in, self.K)
+        assert not self.packed[:, rb:].any()
+        tail_bits = rb * 8 - n_pairs * B
+        if tail_bits:
+            assert not np.any(self.packed[:, rb - 1] >> (8 - tail_bits))
+        return int(diff.sum()), int(exempt.sum()), idx_gpu.size
+
+    def check_decode(self):
+        s = np.ones(self.d_in) if self.s is None else self.s.astype(np.float64)
+        ref_bits, ref64 = self.orc.decode(self.enc["packed"], self.enc["row_norm"], self.block, self.cb_host, self.s,
+                                          self.signs, self.sigma, self.d_in, want_f64=True)
+        ulps = np.abs(_bf16_ordered(self.what) - _bf16_ordered(ref_bits))
+        got = self.orc.bf16_to_f32(self.what).astype(np.float64)
+        yhat = self.cb_host[self.enc["idx"]].astype(np.float64) * self.sigma.astype(np.float64)[None, :, None]
+        blk = np.sqrt((yhat.reshape(len(self.rows), -1, self.block) ** 2).sum(2))  # |yhat_block|_2
+        abs_tol = 2.0**-21 * np.repeat(blk, self.block, axis=1) * self.enc["row_norm"].astype(np.float64)[:, None] / s
+        ok = (ulps <= 1) | (np.abs(got - ref64) <= abs_tol + 2.0**-8 * np.abs(ref64) * 0.51)
+        assert np.all(ok), f"{int((~ok).sum())} decoded weights out of tolerance"
+        return float((ulps == 0).mean()), int((ulps > 1).sum())
+
+    def check_distortion(self):
+        ref = self.orc.distortion(_to_bits(self.Wd), self.what_full, self.act)
+        np.testing.assert_allclose(self.out4, ref, rtol=1e-9)
+
+    def check_all(self, expect_bit_identical=True):
+        self.check_calibration()
+        same_z, same_r = self.check_front_half()
+        if expect_bit_identical:
+            assert same_z and same_r
+        n_diff, n_exempt, n = self.check_indices()
+        exact_frac, n_far = self.check_decode()
+        self.check_distortion()
+        assert exact_frac > 0.98
+        assert self.status_word == 0
+        return dict(mismatches=n_diff, exempt=n_exempt, pairs=n, decode_exact=exact_frac, decode_gt1ulp=n_far)
+
+
+# ------------------------------------------------------------------------------------------------
+def test_cfg0_full(orc):
+    """Configuration 0: W[1024,1024] f32, alpha 0.5, block 128, K 256 -- every row checked."""
+    spec = synth.workload("cfg0")
+    W = synth.make_weight(spec, spec.matrices[0], synth.matrix_seed(spec, 0, 0))
+    act = synth.make_act_rms(spec, 1024, 1).numpy()
+    rep = Case(orc, W, act, spec.alpha, spec.block, spec.K).check_all()
+    print("cfg0", rep)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("block", [2, 4, 8, 16, 32, 64, 128, 256, 512, 1024])
+def test_block_sizes(orc, block, dtype):
+    W, act = _make(37, 2048, dtype, 100 + block)
+    Case(orc, W, act, 0.3, block, 256).check_all()
+
+
+@pytest.mark.parametrize("K", [2, 4, 16, 64, 128, 1024, 2048, 4096])
+def test_codebook_sizes(orc, K):
+    W, act = _make(33, 1024, torch.bfloat16, 200 + K)
+    Case(orc, W, act, 0.3, 128, K).check_all()
+
+
+@pytest.mark.parametrize("d_out,d_in,block", [(1, 2, 2), (3, 4, 4), (5, 6, 2), (1, 8, 8), (7, 24, 8), (3, 40, 8),
+                                              (1025, 64, 64), (2, 192, 64), (9, 1152, 128), (3, 16384, 1024)])
+def test_ragged_shapes(orc, d_out, d_in, block):
+    """Rows shorter than a thread's 32 elements, rows that are not a multiple of 8 long (element-wise
+    load path), more rows than one wave of the grid, the longest supported row."""
+    W, act = _make(d_out, d_in, torch.float32, d_out * 7 + d_in)
+    Case(orc, W, act, 0.5, block, 64).check_all()
+
+
+def test_strided_and_misaligned_rows(orc):
+    base, act = _make(16, 520, torch.bfloat16, 5)
+    base = base.to(DEV)
+    W = base[:, 3:515]  # row stride 520, rows start 6 bytes off a 16-byte boundary
+    assert W.stride(0) == 520 and W.data_ptr() % 16 == 6
+    Case(orc, W, act[3:515], 0.3, 128, 256, packed_stride=720).check_all()
+    W = base[:, 8:520]  # aligned, strided
+    Case(orc, W, act[8:520], 0.3, 128, 256).check_all()
+
+
+def test_no_channel_scaling_and_brute_force_flag(orc):
+    W, act = _make(64, 1024, torch.bfloat16, 11)
+    a = Case(orc, W, act, 0.0, 128, 2048)
+    a.check_all()
+    b = Case(orc, W, act, 0.0, 128, 2048, flags=q.FLAG_BRUTE_FORCE)
+    b.check_all()
+    B = 11
+    ia = np.stack([orc.unpack_row(r, 512, B) for r in a.packed])
+    ib = np.stack([orc.unpack_row(r, 512, B) for r in b.packed])
+    assert (ia != ib).mean() < 1e-4  # the two searches may differ only on near ties
+
+
+def test_zero_outlier_and_nonfinite_rows(orc):
+    W, act = _make(12, 512, torch.float32, 13, student=False)
+    W[2] = 0
+    W[5, 17] = 3.0e4  # one huge entry: its block's points leave the table's [-8, 8) square
+    c = Case(orc, W, act, 0.0, 128, 256)
+    c.check_all()
+    assert c.norm[2] == 0 and not orc.bf16_to_f32(c.what_full[2]).any()
+    W[7, 100] = float("inf")
+    W[9, 3] = float("nan")
+    c = Case(orc, W, act, 0.0, 128, 256)
+    assert c.status_word == 1 and q.status_to_error(c.status_word) == q.ERR_NONFINITE
+    assert c.enc["status"] == orc.ORC_ERR_NONFINITE
+    ok = [r for r in range(12) if r not in (7, 9)]  # the other rows are unaffected
+    B, n_pairs = 8, 256
+    idx_gpu = np.stack([orc.unpack_row(c.packed[r], n_pairs, B) for r in ok])
+    exempt = (c.enc["d2_second"][ok] - c.enc["d2_best"][ok]) < 1e-6 * c.enc["d2_second"][ok]
+    assert not np.any((idx_gpu != c.enc["idx"][ok]) & ~exempt)
+
+
+def test_extreme_z_falls_back_to_exhaustive_search(orc):
+    """sigma far too small drives every point outside the table; the exhaustive fallback must agree."""
+    W, act = _make(6, 256, torch.float32, 17, student=False)
+    cb_host, cb = _codebook(orc, 256)
+    signs = q.make_signs(q.DEFAULT_SIGN_SEED, 256)
+    sigma = np.full(128, 1e-3, np.float32)
+    p = q.make_params(W.to(DEV), 6, 256, 64, 256)
+    packed = torch.zeros((6, p.packed_row_stride), dtype=torch.uint8, device=DEV)
+    norm = torch.empty(6, dtype=torch.float32, device=DEV)
+    q.encode(W.to(DEV), p, None, torch.from_numpy(signs).to(DEV), torch.from_numpy(sigma).to(DEV), cb, packed, norm)
+    enc = orc.encode(W.numpy(), 64, cb_host, None, signs, sigma, packed_row_stride=p.packed_row_stride, diagnostics=True)
+    assert np.abs(enc["z"]).max() > 8
+    idx_gpu = np.stack([orc.unpack_row(r, 128, 8) for r in packed.cpu().numpy()])
+    exempt = (enc["d2_second"] - enc["d2_best"]) < 1e-6 * enc["d2_second"]
+    assert not np.any((idx_gpu != enc["idx"]) & ~exempt)
+
+
+@pytest.mark.parametrize("name,mid", [("cfg3", 0), ("cfg3", 4), ("cfg3", 6), ("cfg1", 6), ("cfg2", 1)])
+def test_full_size_matrices_sampled_rows(orc, name, mid):
+    """Benchmark-size matrices in the benchmark's launch configuration (whole matrix on the device,
+    generated there); the oracle checks a spread of sampled rows."""
+    spec = synth.workload(name)
+    m = spec.matrices[mid]
+    W = synth.make_weight(spec, m, synth.matrix_seed(spec, 0, mid), device=DEV)
+    act = synth.make_act_rms(spec, m.d_in, 3, device=DEV).cpu().numpy()
+    rows = np.unique(np.concatenate([[0, 1, m.d_out - 1], np.linspace(0, m.d_out - 1, 45).astype(int)]))
+    rep = Case(orc, W, act, spec.alpha, spec.block, spec.K, row_sel=rows).check_all()
+    print(name, m.name, rep)
+
+
+def test_encode_decode_are_deterministic(orc):
+    W, act = _make(300, 2048, torch.bfloat16, 23)
+    a = Case(orc, W, act, 0.3, 128, 2048)
+    b = Case(orc, W, act, 0.3, 128, 2048)
+    assert np.array_equal(a.packed, b.packed) and np.array_equal(a.norm, b.norm)
+    assert np.array_equal(a.what_full, b.what_full) and np.array_equal(a.sigma_gpu, b.sigma_gpu)
+
+
+def test_empty_matrix(orc):
+    cb_host, cb = _codebook(orc, 64)
+    p = q.make_params(None, 0, 64, 64, 64)
+    dummy = torch.zeros(64, dtype=torch.uint8, device=DEV)
+    signs = torch.ones(64, dtype=torch.int8, device=DEV)
+    sigma = torch.ones(32, dtype=torch.float32, device=DEV)
+    q.encode(dummy, p, None, signs, sigma, cb, dummy, sigma)  # d_out = 0: nothing launched, no error
+    q.decode(dummy, sigma, None, signs, sigma, cb, p, dummy)
+    torch.cuda.synchronize()
