@@ -16,7 +16,7 @@ inline int ilog2(int64_t v) {
     return l;
 }
 
-// Fine binning of one axis: bin = floor(z * kFineScale + kFineOffset), covering [-8, 8).
+// Fine binning of one axis: bin = clamp(floor(z * kFineScale + kFineOffset), 0, kFineBins - 1).
 constexpr int kFineBins = 4096;
 constexpr double kFineScale = 256.0;
 constexpr double kFineOffset = 2048.0;
@@ -24,7 +24,7 @@ constexpr double kFineOffset = 2048.0;
 // Host form of the search grid: per coarse cell the full candidate list.
 struct CellLists {
     int grid = 0;
-    std::vector<double> edges;        // grid+1 coarse boundaries (z units), edges[0] = -8, edges[grid] = 8
+    std::vector<double> edges;        // grid+1 coarse boundaries (z units); the outermost are +-16384
     std::vector<uint8_t> lut;         // fine bin -> coarse column / row
     std::vector<std::vector<uint16_t>> lists;  // [iy*grid + ix], ascending codeword indices
     int max_list = 0;
@@ -43,13 +43,8 @@ struct SearchTable {
     size_t bytes() const { return lut.size() + cells.size() * 2 + overflow.size() * 2; }
 };
 
-// All codewords whose nearest-neighbour region meets [x0,x1] x [y0,y1] (refine = true), or a
-// superset of those (refine = false, faster).
-void rect_candidates(const double* cb, int K, double x0, double x1, double y0, double y1, bool refine,
-                     std::vector<uint16_t>* out, std::vector<double>* scratch);
-
 int default_grid(int K);
-bool build_cell_lists(const double* cb, int K, int grid, bool refine, CellLists* out);
+bool build_cell_lists(const double* cb, int K, int grid, CellLists* out);
 bool pack_search_table(const CellLists& cl, SearchTable* out);
 
 // grid > 0: exactly that grid (fails if it does not fit); grid == 0: the default grid for K,

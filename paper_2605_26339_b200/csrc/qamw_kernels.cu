@@ -293,9 +293,11 @@ __device__ __noinline__ int search_overflow(const SearchSmem& s, uint2 rec, floa
 }
 
 __device__ __forceinline__ int search_table(const SearchSmem& s, float zx, float zy) {
+    // beyond the table's reach (or NaN): exhaustive scan
+    if (!(fabsf(zx) < 16000.0f && fabsf(zy) < 16000.0f)) return search_exhaustive(s.cb, s.K, zx, zy);
     const float fx = __fmaf_rn(zx, 256.0f, 2048.0f), fy = __fmaf_rn(zy, 256.0f, 2048.0f);
-    if (!(fx >= 0.0f && fx < 4096.0f && fy >= 0.0f && fy < 4096.0f)) return search_exhaustive(s.cb, s.K, zx, zy);
-    const int ix = s.lut[int(fx)], iy = s.lut[int(fy)];
+    const int bx = min(max(int(fx), 0), 4095), by = min(max(int(fy), 0), 4095);
+    const int ix = s.lut[bx], iy = s.lut[by];
     const uint2 rec = s.cells[iy * s.grid + ix];
     if ((rec.x & 0xffffu) == 0xffffu) return search_overflow(s, rec, zx, zy);
     float best = INFINITY;

@@ -7,25 +7,21 @@
 // nearest-neighbour (Voronoi) region meets the cell, hence scanning the list
 // gives the same answer as scanning the codebook.
 //
-// Geometry.  Each axis of [-8, 8) is cut into 4096 fine bins of width 1/256
+// Geometry.  Each axis is cut into 4096 fine bins of width 1/256 over [-8, 8)
 // (powers of two, so the device's fma(z, 256, 2048) is exact up to its final
-// rounding).  A byte look-up table maps a fine bin to one of `grid` coarse
-// columns; column boundaries sit on fine-bin edges, near the quantiles of
-// N(0, 2), which is the marginal of the high-rate optimal point density
-// f^(1/2) of a unit circular Gaussian source -- so every coarse cell holds
-// about the same number of codewords.  Points outside [-8, 8)^2 are not covered
-// and are scanned exhaustively by the device.
+// rounding); the first and last bin also take everything beyond (the device
+// clamps the bin index), out to |z| < 16384.  A byte look-up table maps a fine
+// bin to one of `grid` coarse columns.  Column boundaries sit on fine-bin
+// edges: the inner ones near the quantiles of N(0, 2) -- the marginal of the
+// high-rate optimal point density f^(1/2) of a unit circular Gaussian source,
+// so that every inner cell holds about the same number of codewords -- followed
+// by a few geometrically widening tail columns for heavy-tailed inputs.
 //
-// Construction for one cell Q (enlarged by a margin that covers the rounding of
-// the device's f32 index computation):
-//   1. U = min_i max_{z in Q} |z - c_i|^2.  Whatever z in Q is, its nearest
-//      codeword is no farther than sqrt(U), so a codeword whose minimum
-//      distance to Q exceeds U can never win inside Q.  This gives a superset A.
-//   2. For every i in A the rectangle is clipped by the half-planes
-//      |z - c_i|^2 <= |z - c_j|^2 (j in A, relaxed by a small slack); i stays
-//      iff the clipped polygon is not empty, i.e. iff the region of i really
-//      meets Q.  Competitors outside A cannot be nearest in Q, so clipping
-//      against A alone is exact.
+// Construction.  The Voronoi polygon of every codeword (clipped to the square
+// |z| <= 16384 and relaxed by a small slack, so it can only grow) is obtained by
+// clipping that square with the bisector half-planes of all other codewords.
+// A codeword is listed in a cell iff its polygon meets the cell's rectangle
+// enlarged by a margin that covers the rounding of the device's bin computation.
 #include <algorithm>
 #include <cmath>
 #include <cstring>
@@ -39,21 +35,23 @@ struct Pt {
     double x, y;
 };
 
+constexpr double kFar = 16384.0;  // the table covers |z| < kFar
+
 // Sutherland-Hodgman step: keep the part of convex polygon `in` with a*x + b*y <= c.
-int clip_halfplane(const Pt* in, int n, double a, double b, double c, Pt* out) {
-    int m = 0;
-    for (int i = 0; i < n; ++i) {
+void clip_halfplane(const std::vector<Pt>& in, double a, double b, double c, std::vector<Pt>* out) {
+    out->clear();
+    const size_t n = in.size();
+    for (size_t i = 0; i < n; ++i) {
         const Pt& p = in[i];
         const Pt& q = in[(i + 1) % n];
         double fp = a * p.x + b * p.y - c;
         double fq = a * q.x + b * q.y - c;
-        if (fp <= 0) out[m++] = p;
+        if (fp <= 0) out->push_back(p);
         if ((fp < 0 && fq > 0) || (fp > 0 && fq < 0)) {
             double t = fp / (fp - fq);
-            out[m++] = Pt{p.x + t * (q.x - p.x), p.y + t * (q.y - p.y)};
+            out->push_back(Pt{p.x + t * (q.x - p.x), p.y + t * (q.y - p.y)});
         }
     }
-    return m;
 }
 
 // Quantile of N(0, 2) by bisection on its CDF (1 + erf(x/2))/2; only used to place cell
@@ -67,114 +65,131 @@ double quantile_n02(double p) {
     return 0.5 * (lo + hi);
 }
 
-}  // namespace
-
-static void rect_candidates_rec(const double* cb, int K, double x0, double x1, double y0, double y1, bool refine,
-                                int depth, std::vector<uint16_t>* out, std::vector<double>* scratch) {
-    out->clear();
-    scratch->resize(size_t(K));
-    double U = INFINITY;
-    for (int i = 0; i < K; ++i) {
-        double cx = cb[2 * i], cy = cb[2 * i + 1];
-        double fx = std::max(std::fabs(cx - x0), std::fabs(cx - x1));
-        double fy = std::max(std::fabs(cy - y0), std::fabs(cy - y1));
-        double dmax2 = fx * fx + fy * fy;
-        if (dmax2 < U) U = dmax2;
-        double nx = cx < x0 ? x0 - cx : (cx > x1 ? cx - x1 : 0.0);
-        double ny = cy < y0 ? y0 - cy : (cy > y1 ? cy - y1 : 0.0);
-        (*scratch)[size_t(i)] = nx * nx + ny * ny;
-    }
-    const double lim = U * (1.0 + 1e-12) + 1e-300;
-    std::vector<uint16_t> A;
-    for (int i = 0; i < K; ++i)
-        if ((*scratch)[size_t(i)] <= lim) A.push_back(uint16_t(i));
-    if (!refine || A.size() <= 1) {
-        *out = A;
-        return;
-    }
-    if (A.size() > 24 && depth < 6) {
-        // A large rectangle makes bound 1 loose: cover it by its four quadrants instead and
-        // take the union (a region meets the rectangle iff it meets one of the quadrants).
-        double xm = 0.5 * (x0 + x1), ym = 0.5 * (y0 + y1);
-        std::vector<uint16_t> part, all;
-        const double qx[2][2] = {{x0, xm}, {xm, x1}}, qy[2][2] = {{y0, ym}, {ym, y1}};
-        for (int a = 0; a < 2; ++a)
-            for (int b = 0; b < 2; ++b) {
-                rect_candidates_rec(cb, K, qx[a][0], qx[a][1], qy[b][0], qy[b][1], true, depth + 1, &part, scratch);
-                all.insert(all.end(), part.begin(), part.end());
+// Voronoi polygon of codeword i inside [-kFar, kFar]^2, bisectors relaxed outwards by a slack.
+void voronoi_polygon(const double* cb, int K, int i, std::vector<Pt>* poly, std::vector<Pt>* tmp) {
+    const double cix = cb[2 * i], ciy = cb[2 * i + 1];
+    const double ci2 = cix * cix + ciy * ciy;
+    *poly = {Pt{-kFar, -kFar}, Pt{kFar, -kFar}, Pt{kFar, kFar}, Pt{-kFar, kFar}};
+    double reach2 = 8.0 * kFar * kFar;  // upper bound of the squared distance from c_i to any vertex
+    for (int j = 0; j < K; ++j) {
+        if (j == i) continue;
+        const double cjx = cb[2 * j], cjy = cb[2 * j + 1];
+        const double ddx = cjx - cix, ddy = cjy - ciy;
+        const double d2 = ddx * ddx + ddy * ddy;
+        // the bisector lies at distance |cj - ci| / 2 from c_i: it cannot cut a polygon inside that radius
+        if (d2 > 4.0 * reach2 * (1.0 + 1e-9)) continue;
+        const double cj2 = cjx * cjx + cjy * cjy;
+        const double slack = 1e-11 * (1.0 + ci2 + cj2);
+        // |z-ci|^2 <= |z-cj|^2  <=>  2 z.(cj - ci) <= |cj|^2 - |ci|^2
+        clip_halfplane(*poly, 2 * ddx, 2 * ddy, cj2 - ci2 + slack, tmp);
+        if (tmp->size() != poly->size() || std::memcmp(tmp->data(), poly->data(), poly->size() * sizeof(Pt)) != 0) {
+            poly->swap(*tmp);
+            reach2 = 0.0;
+            for (const Pt& p : *poly) {
+                double ex = p.x - cix, ey = p.y - ciy;
+                reach2 = std::max(reach2, ex * ex + ey * ey);
             }
-        std::sort(all.begin(), all.end());
-        all.erase(std::unique(all.begin(), all.end()), all.end());
-        *out = all;
-        return;
-    }
-    Pt poly[2][72];
-    for (uint16_t i : A) {
-        double cix = cb[2 * i], ciy = cb[2 * i + 1];
-        double ci2 = cix * cix + ciy * ciy;
-        int cur = 0, n = 4;
-        poly[0][0] = Pt{x0, y0};
-        poly[0][1] = Pt{x1, y0};
-        poly[0][2] = Pt{x1, y1};
-        poly[0][3] = Pt{x0, y1};
-        for (uint16_t j : A) {
-            if (j == i) continue;
-            double cjx = cb[2 * j], cjy = cb[2 * j + 1];
-            double cj2 = cjx * cjx + cjy * cjy;
-            // |z-ci|^2 <= |z-cj|^2  <=>  2 z.(cj - ci) <= |cj|^2 - |ci|^2
-            double slack = 1e-11 * (1.0 + ci2 + cj2);
-            n = clip_halfplane(poly[cur], n, 2 * (cjx - cix), 2 * (cjy - ciy), cj2 - ci2 + slack, poly[cur ^ 1]);
-            cur ^= 1;
-            if (n == 0 || n > 64) break;  // n > 64 cannot happen for a convex clip; kept as a guard
         }
-        if (n != 0) out->push_back(i);
+        if (poly->empty()) break;  // cannot happen for distinct codewords; duplicates end up empty
     }
 }
 
-void rect_candidates(const double* cb, int K, double x0, double x1, double y0, double y1, bool refine,
-                     std::vector<uint16_t>* out, std::vector<double>* scratch) {
-    rect_candidates_rec(cb, K, x0, x1, y0, y1, refine, 0, out, scratch);
-}
+}  // namespace
 
 int default_grid(int K) {
     int g = int(std::ceil(2.1 * std::sqrt(double(K)) / 8.0)) * 8;
     return std::max(4, std::min(g, 192));
 }
 
-bool build_cell_lists(const double* cb, int K, int grid, bool refine, CellLists* out) {
-    if (grid < 1 || grid > 255) return false;
-    out->grid = grid;
-    // coarse boundaries (in fine-bin units) near the quantiles of N(0, 2), strictly increasing
+// Coarse boundaries in fine-bin units: edge[0] = 0 < ... < edge[grid] = kFineBins.
+static std::vector<int> make_edges(int grid) {
+    // number of widening tail columns per side (none for tiny grids)
+    const int tails = grid >= 24 ? 3 : (grid >= 12 ? 1 : 0);
+    const int core = grid - 2 * tails;
+    std::vector<double> pos;  // boundaries for z > 0, in z units
+    std::vector<double> inner;
+    for (int i = 1; i < core; ++i) inner.push_back(quantile_n02(double(i) / double(core)));
+    std::vector<double> all(inner);
+    if (tails > 0 && core >= 2) {
+        double last = inner.back();
+        double w = core >= 3 ? (inner[inner.size() - 1] - inner[inner.size() - 2]) * 1.5 : 1.0;
+        std::vector<double> up;
+        double e = last;
+        for (int t = 0; t < tails; ++t) {
+            e += w;
+            w *= 1.5;
+            up.push_back(std::min(e, 7.9 - 0.1 * (tails - 1 - t)));
+        }
+        for (double u : up) all.push_back(u);
+        for (double u : up) all.push_back(-u);
+    }
+    std::sort(all.begin(), all.end());
     std::vector<int> edge(static_cast<size_t>(grid + 1), 0);
     edge[0] = 0;
     edge[size_t(grid)] = kFineBins;
     for (int i = 1; i < grid; ++i) {
-        double q = quantile_n02(double(i) / double(grid));
+        double q = (size_t(i - 1) < all.size()) ? all[size_t(i - 1)] : 7.9;
         int e = int(std::lround(q * kFineScale + kFineOffset));
         e = std::max(e, edge[size_t(i - 1)] + 1);
         e = std::min(e, kFineBins - (grid - i));
         edge[size_t(i)] = e;
     }
+    return edge;
+}
+
+bool build_cell_lists(const double* cb, int K, int grid, CellLists* out) {
+    if (grid < 1 || grid > 255) return false;
+    out->grid = grid;
+    std::vector<int> edge = make_edges(grid);
     out->edges.resize(size_t(grid + 1));
     for (int i = 0; i <= grid; ++i) out->edges[size_t(i)] = (double(edge[size_t(i)]) - kFineOffset) / kFineScale;
+    // the outermost columns also own everything beyond the fine range (the device clamps the bin)
+    out->edges[0] = -kFar;
+    out->edges[size_t(grid)] = kFar;
     out->lut.assign(size_t(kFineBins), 0);
     for (int i = 0; i < grid; ++i)
         for (int f = edge[size_t(i)]; f < edge[size_t(i + 1)]; ++f) out->lut[size_t(f)] = uint8_t(i);
     // 2^-10 of a fine bin covers the rounding of fma(z, 256, 2048) (at most 2^-12 of a bin)
     const double margin = 1.0 / (1024.0 * kFineScale);
     out->lists.assign(size_t(grid) * grid, {});
+    std::vector<Pt> poly, tmp, a, b;
+    auto column_of = [&](double z) {  // coarse column containing z (clamped like the device)
+        double f = std::floor(z * kFineScale + kFineOffset);
+        int fi = int(std::min(double(kFineBins - 1), std::max(0.0, f)));
+        return int(out->lut[size_t(fi)]);
+    };
+    for (int i = 0; i < K; ++i) {
+        voronoi_polygon(cb, K, i, &poly, &tmp);
+        if (poly.empty()) continue;
+        double bx0 = INFINITY, bx1 = -INFINITY, by0 = INFINITY, by1 = -INFINITY;
+        for (const Pt& p : poly) {
+            bx0 = std::min(bx0, p.x); bx1 = std::max(bx1, p.x);
+            by0 = std::min(by0, p.y); by1 = std::max(by1, p.y);
+        }
+        const int ix0 = column_of(bx0 - 2 * margin), ix1 = column_of(bx1 + 2 * margin);
+        const int iy0 = column_of(by0 - 2 * margin), iy1 = column_of(by1 + 2 * margin);
+        for (int iy = iy0; iy <= iy1; ++iy)
+            for (int ix = ix0; ix <= ix1; ++ix) {
+                const double x0 = out->edges[size_t(ix)] - margin, x1 = out->edges[size_t(ix + 1)] + margin;
+                const double y0 = out->edges[size_t(iy)] - margin, y1 = out->edges[size_t(iy + 1)] + margin;
+                clip_halfplane(poly, -1, 0, -x0, &a);          // x >= x0
+                if (a.empty()) continue;
+                clip_halfplane(a, 1, 0, x1, &b);               // x <= x1
+                if (b.empty()) continue;
+                clip_halfplane(b, 0, -1, -y0, &a);             // y >= y0
+                if (a.empty()) continue;
+                clip_halfplane(a, 0, 1, y1, &b);               // y <= y1
+                if (b.empty()) continue;
+                out->lists[size_t(iy) * grid + ix].push_back(uint16_t(i));
+            }
+    }
     out->max_list = 0;
     out->n_candidates = 0;
-    std::vector<double> scratch;
-    for (int iy = 0; iy < grid; ++iy)
-        for (int ix = 0; ix < grid; ++ix) {
-            auto& list = out->lists[size_t(iy) * grid + ix];
-            rect_candidates(cb, K, out->edges[size_t(ix)] - margin, out->edges[size_t(ix + 1)] + margin,
-                            out->edges[size_t(iy)] - margin, out->edges[size_t(iy + 1)] + margin, refine, &list,
-                            &scratch);
-            out->max_list = std::max(out->max_list, int(list.size()));
-            out->n_candidates += int(list.size());
-        }
+    for (const auto& l : out->lists) {
+        if (l.empty()) return false;  // every cell is met by at least one region
+        out->max_list = std::max(out->max_list, int(l.size()));
+        out->n_candidates += int(l.size());
+    }
     return true;
 }
 
@@ -220,7 +235,7 @@ bool choose_search_table(const float* codebook, int K, int grid, size_t budget_b
         }
         CellLists cl;
         SearchTable t;
-        if (build_cell_lists(cb.data(), K, g, true, &cl) && pack_search_table(cl, &t) && t.bytes() <= budget_bytes) {
+        if (build_cell_lists(cb.data(), K, g, &cl) && pack_search_table(cl, &t) && t.bytes() <= budget_bytes) {
             *out = std::move(t);
             return true;
         }

@@ -1,0 +1,126 @@
+"""Whole-model driver over the C ABI: calibrate -> encode -> decode -> distortion for every
+linear weight of a (synthetic) checkpoint.  This is the call a user of the library makes to
+quantise a model; each phase is a plain loop of library calls, one per weight matrix.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+import torch
+
+from . import binding as q
+from . import synth
+
+
+@dataclass
+class MatrixSlot:
+    """Device-resident state of one weight matrix."""
+    name: str
+    d_out: int
+    d_in: int
+    params: q.Params
+    W: torch.Tensor
+    act_rms: torch.Tensor
+    chan_scale: Optional[torch.Tensor]
+    signs: torch.Tensor
+    sigma: torch.Tensor
+    packed: torch.Tensor
+    row_norm: torch.Tensor
+    w_hat: torch.Tensor
+    dist: torch.Tensor  # 4 doubles
+
+
+@dataclass
+class ModelCodec:
+    """All matrices of one workload on one device, plus the shared codebook."""
+    spec: synth.WorkloadSpec
+    device: torch.device
+    codebook: q.Codebook
+    slots: List[MatrixSlot] = field(default_factory=list)
+    workspace: Optional[torch.Tensor] = None
+    status: Optional[torch.Tensor] = None
+    _meta_cache: Dict[int, Tuple[torch.Tensor, torch.Tensor]] = field(default_factory=dict)
+
+    @classmethod
+    def from_synthetic(cls, spec: synth.WorkloadSpec, device, codebook_host: np.ndarray, rank: int = 0,
+                       layers: Optional[List[int]] = None, sign_seed: int = q.DEFAULT_SIGN_SEED) -> "ModelCodec":
+        dev = torch.device(device)
+        with torch.cuda.device(dev):
+            mc = cls(spec, dev, q.Codebook(codebook_host))
+            ws_bytes = 8
+            for layer, mid, m in synth.iter_matrices(spec, layers):
+                seed = synth.matrix_seed(spec, layer, mid, rank)
+                W = synth.make_weight(spec, m, seed, device=dev)
+                act = synth.make_act_rms(spec, m.d_in, seed, device=dev)
+                mc.add_matrix(f"layers.{layer}.{m.name}", W, act, sign_seed)
+                ws_bytes = max(ws_bytes, q.calibrate_workspace_bytes(mc.slots[-1].params))
+            mc.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+            mc.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        return mc
+
+    def add_matrix(self, name: str, W: torch.Tensor, act_rms: torch.Tensor, sign_seed: int = q.DEFAULT_SIGN_SEED):
+        spec, dev = self.spec, self.device
+        d_out, d_in = W.shape
+        p = q.make_params(W, d_out, d_in, spec.block, spec.K)
+        chan_scale = None
+        if spec.alpha:
+            chan_scale = torch.from_numpy(q.channel_scales(act_rms.cpu().numpy(), spec.alpha)).to(dev)
+        if d_in not in self._meta_cache:
+            self._meta_cache[d_in] = torch.from_numpy(q.make_signs(sign_seed, d_in)).to(dev)
+        self.slots.append(MatrixSlot(
+            name, d_out, d_in, p, W, act_rms, chan_scale, self._meta_cache[d_in],
+            torch.empty(d_in // 2, dtype=torch.float32, device=dev),
+            torch.empty((d_out, p.packed_row_stride), dtype=torch.uint8, device=dev),
+            torch.empty(d_out, dtype=torch.float32, device=dev),
+            torch.empty((d_out, d_in), dtype=torch.bfloat16, device=dev),
+            torch.zeros(4, dtype=torch.float64, device=dev)))
+
+    # --- phases: one library call per matrix, asynchronous on the current stream ----------------
+    def calibrate_all(self):
+        for s in self.slots:
+            q.calibrate(s.W, s.params, s.chan_scale, s.signs, s.sigma, self.workspace, self.status)
+
+    def encode_all(self):
+        for s in self.slots:
+            q.encode(s.W, s.params, s.chan_scale, s.signs, s.sigma, self.codebook, s.packed, s.row_norm, self.status)
+
+    def decode_all(self):
+        for s in self.slots:
+            q.decode(s.packed, s.row_norm, s.chan_scale, s.signs, s.sigma, self.codebook, s.params, s.w_hat)
+
+    def distortion_all(self):
+        for s in self.slots:
+            q.distortion(s.W, s.w_hat, s.act_rms, s.params, s.dist)
+
+    def step(self):
+        """One pass of the whole hot path over the model."""
+        self.calibrate_all()
+        self.encode_all()
+        self.decode_all()
+        self.distortion_all()
+
+    # --- accounting -----------------------------------------------------------------------------
+    @property
+    def n_weights(self) -> int:
+        return sum(s.d_out * s.d_in for s in self.slots)
+
+    def algorithmic_bytes(self) -> Tuple[int, int]:
+        """(encode, decode) bytes the codec must move: weights in their dtype, the packed payload
+        and 4-byte row norms."""
+        enc = dec = 0
+        for s in self.slots:
+            payload = s.d_out * q.packed_row_bytes(s.d_in, self.spec.K) + 4 * s.d_out
+            enc += s.d_out * s.d_in * s.W.element_size() + payload
+            dec += s.d_out * s.d_in * 2 + payload
+        return enc, dec
+
+    def kernel_launches_per_step(self) -> int:
+        # calibrate = 2 kernels, encode 1, decode 1, distortion 1 (its memset is not a kernel of ours)
+        return 5 * len(self.slots)
+
+    def totals(self) -> Dict[str, float]:
+        d = torch.stack([s.dist for s in self.slots]).sum(0).cpu().numpy()
+        return {"rho_w": float(np.sqrt(d[0] / d[1])), "rho_o_diag": float(np.sqrt(d[2] / d[3])),
+                "mse": float(d[0] / self.n_weights)}
