@@ -60,6 +60,7 @@ extern "C" {
 #define QAMW_MAX_BLOCK 1024 /* cap of Section 3.3 */
 #define QAMW_MAX_K 4096
 #define QAMW_CALIB_MAX_ROWS 1024 /* "up to 1024 unit-normalized rows" (Section 3.4) */
+#define QAMW_STATIC_SCRATCH_BYTES (16u << 20) /* built-in scratch of qamw_calibrate_static */
 
 typedef struct {
     int32_t d_out, d_in;       /* d_in even, block | d_in */
@@ -156,6 +157,28 @@ size_t qamw_calibrate_workspace_bytes(const qamw_params* p);
 int qamw_calibrate(const void* W, const qamw_params* p, const float* chan_scale, const int8_t* signs,
                    float* sigma_out, void* workspace, size_t workspace_bytes, int32_t* status_out,
                    void* stream);
+
+/* qamw_calibrate for callers that must not allocate device memory.  (The paper has no counterpart
+ * of this entry point: it exists for the way the library is embedded, not for the method.)
+ * Some hosts of this library own the whole device heap themselves, or run inside a region where
+ * cudaMalloc is forbidden or would synchronise the device: an inference server with a fixed memory
+ * plan, a plug-in called between two kernels of somebody else's stream.  They cannot provide the
+ * scratch buffer that qamw_calibrate wants.  This variant takes the same inputs and writes the same
+ * sigma_out, but keeps its partial sums in an array of QAMW_STATIC_SCRATCH_BYTES (16 MiB) that is
+ * compiled into the library.  Every device that loads the library holds that array until the
+ * process exits.  The call itself allocates nothing: no cudaMalloc, no cudaFree, no allocating
+ * library routine.
+ *   - Shapes whose scratch need (qamw_calibrate_workspace_bytes) exceeds the array are refused with
+ *     QAMW_ERR_NOMEM and a message in qamw_last_cuda_error(); nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.  Later calls only launch.
+ *   - All calls on a device share the one array, and it keeps what the last call left there.  No
+ *     part of it has to be zero on entry, so nothing is cleared; but two calls whose kernels may
+ *     run at the same time on one device (different streams, different host threads) overwrite each
+ *     other's partial sums: order them on one stream or with events.
+ * Arguments, results and error codes are otherwise those of qamw_calibrate. */
+int qamw_calibrate_static(const void* W, const qamw_params* p, const float* chan_scale, const int8_t* signs,
+                          float* sigma_out, int32_t* status_out, void* stream);
 
 /* Section 3.1 steps 1-6 (after Section B.2 scaling) for all rows.  Writes packed_out
  * [d_out, packed_row_stride] bytes, row_norm_out [d_out] f32 and ORs bit 0 into *status_out

@@ -29,7 +29,7 @@ EXPORTED = [
     "qamw_train_codebook", "qamw_channel_scales", "qamw_make_signs", "qamw_block_size_rule",
     "qamw_packed_row_bytes", "qamw_bpw", "qamw_status_to_error", "qamw_codebook_create",
     "qamw_codebook_destroy", "qamw_codebook_table_info", "qamw_search_table_build",
-    "qamw_calibrate_workspace_bytes", "qamw_calibrate", "qamw_encode", "qamw_rotate", "qamw_decode",
+    "qamw_calibrate_workspace_bytes", "qamw_calibrate", "qamw_calibrate_static", "qamw_encode", "qamw_rotate", "qamw_decode",
     "qamw_distortion", "qamw_last_cuda_error",
 ]
 
@@ -76,6 +76,7 @@ def lib() -> C.CDLL:
         L.qamw_calibrate_workspace_bytes.argtypes = [C.POINTER(Params)]
         L.qamw_calibrate_workspace_bytes.restype = sz
         L.qamw_calibrate.argtypes = [vp, C.POINTER(Params), vp, vp, vp, vp, sz, vp, vp]
+        L.qamw_calibrate_static.argtypes = [vp, C.POINTER(Params), vp, vp, vp, vp, vp]
         L.qamw_encode.argtypes = [vp, C.POINTER(Params), vp, vp, vp, vp, vp, vp, vp, vp]
         L.qamw_rotate.argtypes = [vp, C.POINTER(Params), vp, vp, vp, vp, vp, vp]
         L.qamw_decode.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Params), vp, vp]
@@ -239,6 +240,21 @@ def calibrate(W: torch.Tensor, p: Params, chan_scale, signs, sigma_out: torch.Te
     _check("qamw_calibrate", lib().qamw_calibrate(_dp(W), C.byref(p), _dp(chan_scale), _dp(signs), _dp(sigma_out),
                                                  _dp(workspace), workspace.numel() * workspace.element_size(),
                                                  _dp(status), _stream(stream)))
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def calibrate_static(W: torch.Tensor, p: Params, chan_scale, signs, sigma_out: torch.Tensor,
+                     status: Optional[torch.Tensor] = None, stream=None):
+    """qamw_calibrate without a caller-provided workspace: for hosts that may not allocate device
+    memory.  The partial sums live in a 16 MiB array built into the library; calls on one device
+    share it, so calls that could overlap on the GPU must be ordered by the caller."""
+    rc = lib().qamw_calibrate_static(_dp(W), C.byref(p), _dp(chan_scale), _dp(signs), _dp(sigma_out), _dp(status),
+                                     _stream(stream))
+    if rc == ERR_NOMEM:
+        raise QamwError("qamw_calibrate_static", rc, lib().qamw_last_cuda_error().decode())
+    _check("qamw_calibrate_static", rc)
 
 
 def encode(W: torch.Tensor, p: Params, chan_scale, signs, sigma, cb: Codebook, packed_out: torch.Tensor,

@@ -18,6 +18,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "qamw_internal.h"
@@ -948,6 +949,59 @@ extern "C" int qamw_calibrate(const void* W, const qamw_params* p, const float* 
     calibrate_finish_kernel<<<(n_pairs + 127) / 128, 128, 0, st>>>(a.partial, c.total_groups, c.pair_stride, n_pairs,
                                                                     p->d_in, sigma_out);
     return finish_launch("calibrate_finish_kernel");
+}
+
+// ---------------------------------------------------------------------------------------------
+// calibration for callers that cannot allocate device memory
+// ---------------------------------------------------------------------------------------------
+
+// Scratch of qamw_calibrate_static.  It is part of the library image: every device that loads the
+// library holds these bytes until the process exits.  In host code the name below is only a handle
+// for cudaGetSymbolAddress; it is never passed to a kernel as if it were a device address.
+static __device__ __align__(256) unsigned char g_static_calib_scratch[QAMW_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_scratch_mutex;
+void* g_static_scratch_ptr[kMaxDevices] = {};  // device address of the array, per device ordinal
+}  // namespace
+
+extern "C" int qamw_calibrate_static(const void* W, const qamw_params* p, const float* chan_scale,
+                                     const int8_t* signs, float* sigma_out, int32_t* status_out, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    const size_t need = qamw_calibrate_workspace_bytes(p);
+    if (need > size_t(QAMW_STATIC_SCRATCH_BYTES)) {
+        std::snprintf(g_last_error, sizeof(g_last_error),
+                      "qamw_calibrate_static: this shape needs %zu bytes of scratch, the built-in array holds %zu",
+                      need, size_t(QAMW_STATIC_SCRATCH_BYTES));
+        return QAMW_ERR_NOMEM;
+    }
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        set_cuda_error("qamw_calibrate_static: cudaGetDevice", int(e == cudaSuccess ? cudaErrorInvalidDevice : e));
+        return QAMW_ERR_CUDA;
+    }
+    void* scratch = nullptr;
+    {
+        // first call on this device: look up where the array lives in this device's memory
+        std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+        if (!g_static_scratch_ptr[dev]) {
+            void* ptr = nullptr;
+            e = cudaGetSymbolAddress(&ptr, g_static_calib_scratch);
+            if (e != cudaSuccess || !ptr) {
+                set_cuda_error("qamw_calibrate_static: cudaGetSymbolAddress", int(e));
+                return QAMW_ERR_CUDA;
+            }
+            g_static_scratch_ptr[dev] = ptr;
+        }
+        scratch = g_static_scratch_ptr[dev];
+    }
+    // Nothing in the scratch has to start at zero: every word the reduction reads is written
+    // earlier in the same call, so the previous call's contents are simply overwritten.
+    return qamw_calibrate(W, p, chan_scale, signs, sigma_out, scratch, size_t(QAMW_STATIC_SCRATCH_BYTES), status_out,
+                          stream);
 }
 
 extern "C" int qamw_decode(const uint8_t* packed, const float* row_norm, const float* chan_scale, const int8_t* signs,
