@@ -1,17 +1,27 @@
 // CUDA kernels (sm_100a) and device-side entry points of libqamw.
 //
-// Thread geometry shared by every row kernel.  A row of d_in elements is owned by one
-// "group" of TG threads (a whole number of warps); a thread block holds GROUPS such groups,
-// each working on its own row, and the grid is persistent (rows are strided over all groups).
-// A thread keeps 32 elements of its row in registers as four "octets" of eight contiguous
-// elements.  With L = max(1, b/32) threads per Hadamard block of size b, thread l of a block
-// owns octets l, l+L, l+2L, l+3L of that block (for b < 32 a thread owns 32 contiguous
-// elements, i.e. several whole blocks).  The butterfly stages h = 1, 2, 4 then stay inside an
-// octet, stages 8 .. 4L are exchanged with warp shuffles (L <= 32, so never across warps) and
-// the last two stages (b/4, b/2) combine the thread's own octets.  Stages are always executed
-// in ascending order of h, which is what makes the f32 result reproducible bit for bit.
-// The thread owns the same columns in every row, so the per-column factors (channel scale
-// times sign, pair scales) live in registers for the whole kernel.
+// Thread geometry shared by the row kernels (encode, decode, calibrate, rotate).
+//   * A row of d_in elements is owned by one "group" of TG threads (whole warps); a thread block
+//     holds several groups, each on its own row, and the grid is persistent: rows are strided
+//     over all groups of all blocks.
+//   * Thread t of a group owns the 32 contiguous elements [32 t, 32 t + 32) of the row as four
+//     "octets" of eight elements, kept in registers as 4 x 4 packed f32 pairs, so the thread reads
+//     (encode) or writes (decode) 16-byte pieces and the per-column constants of its columns stay
+//     in registers for the whole kernel.
+//   * Walsh-Hadamard butterflies of a block of b elements: stages h = 1, 2, 4 work inside an octet,
+//     h = 8, 16 between the thread's octets, and for b > 32 the stages h = 32 ... b/2 pair the
+//     L = b/32 threads of the block (L <= 32, never across warps).  Stages always run in ascending
+//     order of h with one f32 rounding per output, which makes the result reproducible bit for bit.
+//   * A cross-thread stage is a "half exchange": instead of both threads fetching all 32 partner
+//     values, each thread sends two of its octets and receives two, then computes both outputs
+//     (a + c, a - c) of the 16 butterflies whose inputs it now holds.  That halves the shuffles;
+//     the price is that the stage swaps the roles of a lane bit and an octet-slot bit, so after
+//     the rotation a thread holds other octets of the block than before (octet_after()).  For the
+//     first two cross stages the threads with the lane bit set load their octets in swapped
+//     register slots, which makes "keep slot 0, send slot 1" the same code for both partners.
+//   * Shared-memory reads are what limits these kernels on B200 (random 8-byte reads replay on
+//     bank conflicts), hence: the codebook is stored in several bank-separated copies and every
+//     lane reads the copy of its own banks.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -40,16 +50,59 @@ namespace {
 constexpr int kMaxThreads = 512;   // threads per block (register budget: 128 per thread)
 constexpr int kMaxGroups = 15;     // named barriers 1..15
 constexpr unsigned kFull = 0xffffffffu;
+constexpr size_t kSmemLimit = 227 * 1024;
 
 struct RowGeom {
     int d_out, d_in;
     int log2b;        // log2 of the Hadamard block
     int tg;           // threads per group (multiple of 32)
     int groups;       // groups per thread block
-    int vec;          // rows can be read with 16-byte loads
+    int vec;          // rows can be moved with 16-byte accesses
     int w_bf16;       // 1 = bf16 weights, 0 = f32
     long long w_row_stride;  // elements
 };
+
+// ---------------------------------------------------------------------------------------------
+// packed f32x2 arithmetic: two IEEE f32 operations (round to nearest even, each half rounded on
+// its own) in one instruction; it halves the issue slots of the butterflies.
+// ---------------------------------------------------------------------------------------------
+typedef unsigned long long f32x2;
+
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 shfl_xor2(f32x2 v, int lane_mask) {
+    float lo, hi;
+    unpack2(v, lo, hi);
+    lo = __shfl_xor_sync(kFull, lo, lane_mask);
+    hi = __shfl_xor_sync(kFull, hi, lane_mask);
+    return pack2(lo, hi);
+}
 
 // ---------------------------------------------------------------------------------------------
 // small device helpers
@@ -65,69 +118,145 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
-// Element offset of octet m of this thread, given its index inside the group.
+// Which octet of the row (in units of 8 elements) sits in register slot r of thread tid_g:
+//   octet_before: when the row enters the rotation;  octet_after: after all butterfly stages.
+// S = number of cross-thread stages, L = 2^S threads per block.  Cross stage j exchanges on slot
+// bit (j & 1); afterwards lane bit j selects bit j of the octet index inside the block and the
+// slot bits select its two top bits, so the L threads of a block write L consecutive octets.
 template <int LOG2B_T>
-__device__ __forceinline__ int octet_offset(int tid_g, int m) {
-    constexpr int L = 1 << (LOG2B_T >= 5 ? LOG2B_T - 5 : 0);
-    if (LOG2B_T >= 5) {
-        const int blk = tid_g / L, l = tid_g % L;
-        return (blk << LOG2B_T) + 8 * (l + L * m);
+struct Layout {
+    static constexpr int S = LOG2B_T > 5 ? LOG2B_T - 5 : 0;
+    static constexpr int L = 1 << S;
+    __device__ static __forceinline__ int octet_before(int tid_g, int r) {
+        int flip = 0;
+        if (S >= 1) flip |= tid_g & 1;
+        if (S >= 2) flip |= tid_g & 2;
+        return 4 * tid_g + (r ^ flip);
     }
-    return tid_g * 32 + 8 * m;
-}
+    __device__ static __forceinline__ int octet_after(int tid_g, int r) {
+        if (S == 0) return 4 * tid_g + r;
+        const int q = tid_g & (L - 1), blk = tid_g >> S;
+        const int hi = (S & 1) ? (((r >> 1) & 1) | ((r & 1) << 1)) : r;
+        return blk * (4 * L) + q + L * hi;
+    }
+};
 
-// One butterfly (a, c) -> (a + c, a - c), round-to-nearest f32, never fused.
-__device__ __forceinline__ void bfly(float& a, float& c) {
-    float s = __fadd_rn(a, c), d = __fsub_rn(a, c);
+// (a, c) -> (a + c, a - c) on two packed registers.
+__device__ __forceinline__ void bfly2(f32x2& a, f32x2& c) {
+    const f32x2 s = add2(a, c), d = sub2(a, c);
     a = s;
     c = d;
 }
 
-// Unnormalised Walsh-Hadamard butterfly of the thread's 4 x 8 elements, stages ascending.
-// LOG2B_T >= 5: block size 2^LOG2B_T known at compile time; LOG2B_T == 0: block size < 32 given
-// at run time (log2b in 1..4).
+// Unnormalised Walsh-Hadamard butterfly of the thread's 4 x 8 elements and, for blocks wider
+// than 32, of the L threads of the block; stages in ascending order.  LOG2B_T >= 5: block size
+// 2^LOG2B_T known at compile time; LOG2B_T == 0: block size 2^log2b_rt <= 16 given at run time.
+// P[r][i] holds elements (2i, 2i+1) of the octet in slot r.
 template <int LOG2B_T>
-__device__ __forceinline__ void fwht_regs(float (&x)[4][8], int log2b_rt, int lane_in_block) {
+__device__ __forceinline__ void fwht_regs(f32x2 (&P)[4][4], int log2b_rt, int tid_g) {
+    typedef Layout<LOG2B_T> Lay;
     const int log2b = LOG2B_T ? LOG2B_T : log2b_rt;
+    if (log2b >= 1) {  // h = 1: inside a packed pair
 #pragma unroll
-    for (int m = 0; m < 4; ++m) {
-        if (log2b >= 1) {
-            bfly(x[m][0], x[m][1]); bfly(x[m][2], x[m][3]); bfly(x[m][4], x[m][5]); bfly(x[m][6], x[m][7]);
-        }
-        if (log2b >= 2) {
-            bfly(x[m][0], x[m][2]); bfly(x[m][1], x[m][3]); bfly(x[m][4], x[m][6]); bfly(x[m][5], x[m][7]);
-        }
-        if (log2b >= 3) {
-            bfly(x[m][0], x[m][4]); bfly(x[m][1], x[m][5]); bfly(x[m][2], x[m][6]); bfly(x[m][3], x[m][7]);
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float a, c;
+                unpack2(P[r][i], a, c);
+                P[r][i] = pack2(__fadd_rn(a, c), __fsub_rn(a, c));
+            }
+    }
+    if (log2b >= 2) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            bfly2(P[r][0], P[r][1]);
+            bfly2(P[r][2], P[r][3]);
         }
     }
-    if (LOG2B_T >= 6) {
-        constexpr int L = 1 << (LOG2B_T >= 5 ? LOG2B_T - 5 : 0);
+    if (log2b >= 3) {
 #pragma unroll
-        for (int s = 1; s < L; s <<= 1) {
-            // lower lane: v + p ; upper lane: p - v = fma(v, -1, p) (the product is exact)
-            const float sgn = (lane_in_block & s) ? -1.0f : 1.0f;
-#pragma unroll
-            for (int m = 0; m < 4; ++m)
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    float p = __shfl_xor_sync(kFull, x[m][e], s);
-                    x[m][e] = __fmaf_rn(x[m][e], sgn, p);
-                }
+        for (int r = 0; r < 4; ++r) {
+            bfly2(P[r][0], P[r][2]);
+            bfly2(P[r][1], P[r][3]);
         }
     }
+    // h = 8, 16: between the octets of the thread.  A thread whose slots are swapped for the
+    // first (second) cross stage holds the upper octet in the lower slot, so its sum and
+    // difference change places: out_lo = s*lo + hi, out_hi = lo - s*hi with s = -1 (an fma with
+    // +-1 rounds exactly like the add or subtract it stands for).
+    const float s0 = (Lay::S >= 1 && (tid_g & 1)) ? -1.0f : 1.0f;
+    const float s1 = (Lay::S >= 2 && (tid_g & 2)) ? -1.0f : 1.0f;
     if (log2b >= 4) {
+        const f32x2 sp = pack2(s0, s0), sn = pack2(-s0, -s0);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            bfly(x[0][e], x[1][e]);
-            bfly(x[2][e], x[3][e]);
+        for (int i = 0; i < 4; ++i) {
+            f32x2 a = P[0][i], c = P[1][i];
+            P[0][i] = fma2(a, sp, c);
+            P[1][i] = fma2(c, sn, a);
+            a = P[2][i];
+            c = P[3][i];
+            P[2][i] = fma2(a, sp, c);
+            P[3][i] = fma2(c, sn, a);
         }
     }
     if (log2b >= 5) {
+        const f32x2 sp = pack2(s1, s1), sn = pack2(-s1, -s1);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            bfly(x[0][e], x[2][e]);
-            bfly(x[1][e], x[3][e]);
+        for (int i = 0; i < 4; ++i) {
+            f32x2 a = P[0][i], c = P[2][i];
+            P[0][i] = fma2(a, sp, c);
+            P[2][i] = fma2(c, sn, a);
+            a = P[1][i];
+            c = P[3][i];
+            P[1][i] = fma2(a, sp, c);
+            P[3][i] = fma2(c, sn, a);
+        }
+    }
+    // Cross-thread stages j = 0 .. S-1 (h = 32 << j), partner lane = lane ^ (1 << j).
+    // j = 0: slots {0,2} are kept and {1,3} sent; the upper thread loaded its octets swapped, so
+    // this is the same code for both partners.  The sender multiplies by its own sign s, which is
+    // minus the receiver's: with v = -s_r * partner, keep + partner = fma(v, -s_r, keep) and the
+    // difference (lower thread: keep - partner, upper thread: partner - keep) = fma(keep, s_r, v).
+    if (Lay::S >= 1) {
+        const f32x2 sp = pack2(s0, s0), sn = pack2(-s0, -s0);
+#pragma unroll
+        for (int rr = 0; rr < 4; rr += 2)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const f32x2 keep = P[rr][i];
+                const f32x2 v = shfl_xor2(mul2(P[rr + 1][i], sp), 1);
+                P[rr][i] = fma2(v, sn, keep);
+                P[rr + 1][i] = fma2(keep, sp, v);
+            }
+    }
+    if (Lay::S >= 2) {  // j = 1: slots {0,1} kept, {2,3} sent
+        const f32x2 sp = pack2(s1, s1), sn = pack2(-s1, -s1);
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const f32x2 keep = P[rr][i];
+                const f32x2 v = shfl_xor2(mul2(P[rr + 2][i], sp), 2);
+                P[rr][i] = fma2(v, sn, keep);
+                P[rr + 2][i] = fma2(keep, sp, v);
+            }
+    }
+#pragma unroll
+    for (int j = 2; j < Lay::S; ++j) {  // later stages: kept and sent slots are selected per thread
+        const bool upper = (tid_g >> j) & 1;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const int ra = (j & 1) ? t : 2 * t;            // slot with partition bit 0
+            const int rb = (j & 1) ? t + 2 : 2 * t + 1;    // slot with partition bit 1
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const f32x2 keep = upper ? P[rb][i] : P[ra][i];
+                const f32x2 send = upper ? P[ra][i] : P[rb][i];
+                const f32x2 got = shfl_xor2(send, 1 << j);
+                const f32x2 a = upper ? got : keep, c = upper ? keep : got;
+                P[ra][i] = add2(a, c);
+                P[rb][i] = sub2(a, c);
+            }
         }
     }
 }
@@ -142,23 +271,23 @@ template <bool BF16, int LOG2B_T>
 __device__ __forceinline__ void load_row(RawRow<BF16>& raw, const void* W, long long row, const RowGeom& g, int tid_g) {
     const char* base = static_cast<const char*>(W) + row * g.w_row_stride * (BF16 ? 2 : 4);
 #pragma unroll
-    for (int m = 0; m < 4; ++m) {
-        const int e0 = octet_offset<LOG2B_T>(tid_g, m);
+    for (int r = 0; r < 4; ++r) {
+        const int e0 = 8 * Layout<LOG2B_T>::octet_before(tid_g, r);
         if (g.vec) {
             if (e0 < g.d_in) {
                 const uint4* p = reinterpret_cast<const uint4*>(base + size_t(e0) * (BF16 ? 2 : 4));
                 if (BF16) {
-                    raw.v[m] = __ldg(p);
+                    raw.v[r] = __ldg(p);
                 } else {
-                    raw.v[2 * m] = __ldg(p);
-                    raw.v[2 * m + 1] = __ldg(p + 1);
+                    raw.v[2 * r] = __ldg(p);
+                    raw.v[2 * r + 1] = __ldg(p + 1);
                 }
             } else {
                 if (BF16) {
-                    raw.v[m] = make_uint4(0, 0, 0, 0);
+                    raw.v[r] = make_uint4(0, 0, 0, 0);
                 } else {
-                    raw.v[2 * m] = make_uint4(0, 0, 0, 0);
-                    raw.v[2 * m + 1] = make_uint4(0, 0, 0, 0);
+                    raw.v[2 * r] = make_uint4(0, 0, 0, 0);
+                    raw.v[2 * r + 1] = make_uint4(0, 0, 0, 0);
                 }
             }
         } else {
@@ -175,10 +304,10 @@ __device__ __forceinline__ void load_row(RawRow<BF16>& raw, const void* W, long 
                 w[e] = bits;
             }
             if (BF16) {
-                raw.v[m] = make_uint4(w[0] | (w[1] << 16), w[2] | (w[3] << 16), w[4] | (w[5] << 16), w[6] | (w[7] << 16));
+                raw.v[r] = make_uint4(w[0] | (w[1] << 16), w[2] | (w[3] << 16), w[4] | (w[5] << 16), w[6] | (w[7] << 16));
             } else {
-                raw.v[2 * m] = make_uint4(w[0], w[1], w[2], w[3]);
-                raw.v[2 * m + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+                raw.v[2 * r] = make_uint4(w[0], w[1], w[2], w[3]);
+                raw.v[2 * r + 1] = make_uint4(w[4], w[5], w[6], w[7]);
             }
         }
     }
@@ -205,41 +334,49 @@ __device__ __forceinline__ void raw_to_float(const RawRow<BF16>& raw, float (&x)
     }
 }
 
-// Per-thread column constants: t_j = f32(s_j) * sign_j (0 beyond the row).
+// Per-thread column constants of the encoder side: t_j = f32(s_j) * sign_j (0 beyond the row),
+// for the columns the thread holds when the row is loaded.
 template <int LOG2B_T>
-__device__ __forceinline__ void load_col_factors(float (&t)[4][8], const float* chan_scale, const int8_t* signs,
+__device__ __forceinline__ void load_col_factors(f32x2 (&t)[4][4], const float* chan_scale, const int8_t* signs,
                                                  int d_in, int tid_g) {
 #pragma unroll
-    for (int m = 0; m < 4; ++m) {
-        const int e0 = octet_offset<LOG2B_T>(tid_g, m);
+    for (int r = 0; r < 4; ++r) {
+        const int e0 = 8 * Layout<LOG2B_T>::octet_before(tid_g, r);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int j = e0 + e;
-            float v = 0.f;
-            if (j < d_in) v = (chan_scale ? chan_scale[j] : 1.0f) * float(signs[j]);
-            t[m][e] = v;
+        for (int i = 0; i < 4; ++i) {
+            float v[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = e0 + 2 * i + h;
+                v[h] = (j < d_in) ? (chan_scale ? chan_scale[j] : 1.0f) * float(signs[j]) : 0.f;
+            }
+            t[r][i] = pack2(v[0], v[1]);
         }
     }
 }
 
 // Scaling, row norm and butterfly of one row held in registers (the arithmetic contract of the
-// encoder, steps x, r, h).  Returns the row norm r; x holds the unnormalised butterfly output.
-// `red` is this group's reduction scratch (one double per warp, two buffers).
+// encoder, steps x, r, h).  Returns the row norm r; P holds the unnormalised butterfly output in
+// the layout of octet_after().  `red` is this group's reduction scratch (one double per warp, two
+// buffers).
 template <bool BF16, int LOG2B_T>
-__device__ __forceinline__ float front_half(const RawRow<BF16>& raw, const float (&t)[4][8], float (&x)[4][8],
-                                            const RowGeom& g, int group, int tid_g, int lane_in_block, double* red,
-                                            int parity) {
+__device__ __forceinline__ float front_half(const RawRow<BF16>& raw, const f32x2 (&t)[4][4], f32x2 (&P)[4][4],
+                                            const RowGeom& g, int group, int tid_g, double* red, int parity) {
+    float x[4][8];
     raw_to_float<BF16>(raw, x);
     double ss = 0.0;
 #pragma unroll
-    for (int m = 0; m < 4; ++m)
+    for (int r = 0; r < 4; ++r)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            x[m][e] = __fmul_rn(x[m][e], t[m][e]);
-            const double xd = double(x[m][e]);
-            ss = fma(xd, xd, ss);
+        for (int i = 0; i < 4; ++i) {
+            P[r][i] = mul2(pack2(x[r][2 * i], x[r][2 * i + 1]), t[r][i]);
+            float a, c;
+            unpack2(P[r][i], a, c);
+            const double ad = double(a), cd = double(c);
+            ss = fma(ad, ad, ss);
+            ss = fma(cd, cd, ss);
         }
-    fwht_regs<LOG2B_T>(x, g.log2b, lane_in_block);
+    fwht_regs<LOG2B_T>(P, g.log2b, tid_g);
     ss = warp_sum(ss);
     const int n_warps = g.tg >> 5;
     double* slot = red + parity * 32;
@@ -256,11 +393,22 @@ __device__ __forceinline__ float inv_norm_factor(float r, int log2b) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// codebook in shared memory: C = 2^log2c copies; entry i of copy c sits at byte (i*C + c) * 8, so
+// the copies of one entry fill consecutive 8-byte bank pairs and a lane that always reads copy
+// (lane mod C) only ever touches its own 16/C bank pairs.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void fill_codebook_copies(float2* dst, const float2* src, int K, int log2c) {
+    const int n = K << log2c;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) dst[i] = __ldg(src + (i >> log2c));
+}
+
+// ---------------------------------------------------------------------------------------------
 // nearest-codeword search
 // ---------------------------------------------------------------------------------------------
 
 struct SearchSmem {
-    const float2* cb;         // K codewords
+    const unsigned char* cb;  // codebook copies, already offset to this lane's copy
+    int cb_shift;             // log2 of the byte distance between consecutive entries (3 + log2c)
     const uint2* cells;       // grid*grid records
     const uint16_t* overflow;
     const uint8_t* lut;       // 4096 bytes
@@ -268,20 +416,28 @@ struct SearchSmem {
     int K;
 };
 
-__device__ __forceinline__ void consider(const float2* cb, int k, float zx, float zy, float& best, int& arg) {
-    const float2 c = cb[k];
+__device__ __forceinline__ float2 codeword(const SearchSmem& s, int k) {
+    return *reinterpret_cast<const float2*>(s.cb + (size_t(k) << s.cb_shift));
+}
+
+// Squared distance in direct form, one rounding per operation: (zx-cx)^2 + (zy-cy)^2.
+__device__ __forceinline__ float dist2(float2 c, float zx, float zy) {
     const float dx = __fsub_rn(zx, c.x), dy = __fsub_rn(zy, c.y);
-    const float d = __fmaf_rn(dy, dy, __fmul_rn(dx, dx));
+    return __fmaf_rn(dy, dy, __fmul_rn(dx, dx));
+}
+
+__device__ __forceinline__ void consider(const SearchSmem& s, int k, float zx, float zy, float& best, int& arg) {
+    const float d = dist2(codeword(s, k), zx, zy);
     if (d < best) {
         best = d;
         arg = k;
     }
 }
 
-__device__ __noinline__ int search_exhaustive(const float2* cb, int K, float zx, float zy) {
+__device__ __noinline__ int search_exhaustive(const SearchSmem& s, float zx, float zy) {
     float best = INFINITY;
     int arg = 0;
-    for (int k = 0; k < K; ++k) consider(cb, k, zx, zy, best, arg);
+    for (int k = 0; k < s.K; ++k) consider(s, k, zx, zy, best, arg);
     return arg;
 }
 
@@ -289,26 +445,41 @@ __device__ __noinline__ int search_overflow(const SearchSmem& s, uint2 rec, floa
     const int off = int(rec.x >> 16), cnt = int(rec.y & 0xffffu);
     float best = INFINITY;
     int arg = 0;
-    for (int i = 0; i < cnt; ++i) consider(s.cb, int(s.overflow[off + i]), zx, zy, best, arg);
+    for (int i = 0; i < cnt; ++i) consider(s, int(s.overflow[off + i]), zx, zy, best, arg);
     return arg;
 }
 
 __device__ __forceinline__ int search_table(const SearchSmem& s, float zx, float zy) {
     // beyond the table's reach (or NaN): exhaustive scan
-    if (!(fabsf(zx) < 16000.0f && fabsf(zy) < 16000.0f)) return search_exhaustive(s.cb, s.K, zx, zy);
+    if (!(fmaxf(fabsf(zx), fabsf(zy)) < 16000.0f)) return search_exhaustive(s, zx, zy);
     const float fx = __fmaf_rn(zx, 256.0f, 2048.0f), fy = __fmaf_rn(zy, 256.0f, 2048.0f);
     const int bx = min(max(int(fx), 0), 4095), by = min(max(int(fy), 0), 4095);
     const int ix = s.lut[bx], iy = s.lut[by];
     const uint2 rec = s.cells[iy * s.grid + ix];
-    if ((rec.x & 0xffffu) == 0xffffu) return search_overflow(s, rec, zx, zy);
-    float best = INFINITY;
-    int arg = 0;
-    consider(s.cb, int(rec.x & 0xffffu), zx, zy, best, arg);
-    consider(s.cb, int(rec.x >> 16), zx, zy, best, arg);
-    consider(s.cb, int(rec.y & 0xffffu), zx, zy, best, arg);
-    consider(s.cb, int(rec.y >> 16), zx, zy, best, arg);
+    const int k0 = int(rec.x & 0xffffu);
+    if (k0 == 0xffff) return search_overflow(s, rec, zx, zy);
+    const int k1 = int(rec.x >> 16), k2 = int(rec.y & 0xffffu), k3 = int(rec.y >> 16);
+    // The list is ascending and padded by repeating its last entry: a repeated slot needs no
+    // second read, its distance is the one just computed.
+    const float d0 = dist2(codeword(s, k0), zx, zy);
+    float d1 = d0;
+    if (k1 != k0) d1 = dist2(codeword(s, k1), zx, zy);
+    float d2 = d1;
+    if (k2 != k1) d2 = dist2(codeword(s, k2), zx, zy);
+    float d3 = d2;
+    if (k3 != k2) d3 = dist2(codeword(s, k3), zx, zy);
+    // lowest slot (= lowest index) among equal distances
+    float best = d0;
+    int arg = k0;
+    if (d1 < best) { best = d1; arg = k1; }
+    if (d2 < best) { best = d2; arg = k2; }
+    if (d3 < best) { best = d3; arg = k3; }
     return arg;
 }
+
+// Position of pair k in the index staging row: 16 halfwords of padding after every 64 pairs keep
+// the 8-byte stores of a warp (eight runs of 32 bytes, 128 bytes apart) on distinct banks.
+__device__ __forceinline__ int stage_pos(int k) { return k + ((k >> 6) << 4); }
 
 // ---------------------------------------------------------------------------------------------
 // encode kernel
@@ -320,10 +491,12 @@ struct EncodeArgs {
     const float* chan_scale;
     const int8_t* signs;
     const float* sigma;
-    const uint4* blob;       // codebook + table, as laid out by qamw_codebook_create
-    int blob_bytes;
-    int off_cells, off_overflow, off_lut;
+    const float2* codebook;  // device, K entries
+    const uint4* table;      // cells | overflow | lut, as laid out by qamw_codebook_create
+    int table_bytes;
+    int off_overflow, off_lut;  // byte offsets inside the table
     int K, log2K, grid;
+    int log2c;               // log2 of the number of codebook copies in shared memory
     int brute;
     uint8_t* packed;
     long long packed_row_stride;  // bytes
@@ -337,39 +510,44 @@ template <bool BF16, int LOG2B_T>
 __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
     const RowGeom& g = a.g;
-    // shared memory: [blob][red: groups x 64 doubles][idx: groups x idx_stride u16]
+    // shared memory: [codebook copies][table][red: groups x 64 doubles][idx: groups x idx_stride u16]
+    const int cb_bytes = (a.K * 8) << a.log2c;
+    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
+    unsigned char* table = smem + cb_bytes;
     {
-        uint4* dst = reinterpret_cast<uint4*>(smem);
-        for (int i = threadIdx.x; i < a.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(a.blob + i);
+        uint4* dst = reinterpret_cast<uint4*>(table);
+        for (int i = threadIdx.x; i < a.table_bytes / 16; i += blockDim.x) dst[i] = __ldg(a.table + i);
     }
-    const int blob_pad = (a.blob_bytes + 15) & ~15;
-    double* red_all = reinterpret_cast<double*>(smem + blob_pad);
-    uint16_t* idx_all = reinterpret_cast<uint16_t*>(smem + blob_pad + g.groups * 64 * sizeof(double));
+    const int table_pad = (a.table_bytes + 15) & ~15;
+    double* red_all = reinterpret_cast<double*>(table + table_pad);
+    uint16_t* idx_all = reinterpret_cast<uint16_t*>(table + table_pad + g.groups * 64 * sizeof(double));
     __syncthreads();
 
     SearchSmem s;
-    s.cb = reinterpret_cast<const float2*>(smem);
-    s.cells = reinterpret_cast<const uint2*>(smem + a.off_cells);
-    s.overflow = reinterpret_cast<const uint16_t*>(smem + a.off_overflow);
-    s.lut = smem + a.off_lut;
+    s.cb = smem + 8 * (threadIdx.x & ((1 << a.log2c) - 1));
+    s.cb_shift = 3 + a.log2c;
+    s.cells = reinterpret_cast<const uint2*>(table);
+    s.overflow = reinterpret_cast<const uint16_t*>(table + a.off_overflow);
+    s.lut = table + a.off_lut;
     s.grid = a.grid;
     s.K = a.K;
 
     const int group = threadIdx.x / g.tg;
     const int tid_g = threadIdx.x - group * g.tg;
-    const int lane_in_block = (LOG2B_T >= 5) ? (tid_g & ((1 << (LOG2B_T >= 5 ? LOG2B_T - 5 : 0)) - 1)) : 0;
     double* red = red_all + group * 64;
     uint16_t* idx_s = idx_all + size_t(group) * a.idx_stride;
     const int n_pairs = g.d_in >> 1;
 
-    float t[4][8];
+    f32x2 t[4][4];
     load_col_factors<LOG2B_T>(t, a.chan_scale, a.signs, g.d_in, tid_g);
+    // pair positions and reciprocal pair scales of the octets the thread holds after the rotation
+    int k0s[4];
     float q[4][4];
 #pragma unroll
-    for (int m = 0; m < 4; ++m) {
-        const int k0 = octet_offset<LOG2B_T>(tid_g, m) >> 1;
+    for (int r = 0; r < 4; ++r) {
+        k0s[r] = 4 * Layout<LOG2B_T>::octet_after(tid_g, r);
 #pragma unroll
-        for (int p = 0; p < 4; ++p) q[m][p] = (k0 + p < n_pairs) ? float(1.0 / double(a.sigma[k0 + p])) : 0.f;
+        for (int p = 0; p < 4; ++p) q[r][p] = (k0s[r] + p < n_pairs) ? float(1.0 / double(a.sigma[k0s[r] + p])) : 0.f;
     }
 
     const long long row_step = (long long)gridDim.x * g.groups;
@@ -384,30 +562,31 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
         const long long next_row = row + row_step;
         if (next_row < g.d_out) load_row<BF16, LOG2B_T>(nxt, a.W, next_row, g, tid_g);
 
-        float x[4][8];
-        const float r = front_half<BF16, LOG2B_T>(raw, t, x, g, group, tid_g, lane_in_block, red, parity);
+        f32x2 P[4][4];
+        const float r = front_half<BF16, LOG2B_T>(raw, t, P, g, group, tid_g, red, parity);
         const bool finite = isfinite(r);
         if (tid_g == 0) {
             a.row_norm[row] = r;
             if (!finite && a.status) atomicOr(a.status, 1);
         }
-        const float gn = (finite && r > 0.f) ? inv_norm_factor(r, g.log2b) : 0.f;
+        const bool live = finite && r > 0.f;  // zero or non-finite rows are encoded as the origin
+        const float gn = live ? inv_norm_factor(r, g.log2b) : 0.f;
+        const f32x2 gn2 = pack2(gn, gn);
 
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            const int k0 = octet_offset<LOG2B_T>(tid_g, m) >> 1;
+        for (int rr = 0; rr < 4; ++rr) {
+            const int k0 = k0s[rr];
             if (k0 < n_pairs) {
                 uint32_t id[4];
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
-                    float zx = 0.f, zy = 0.f;
-                    if (gn != 0.f) {  // zero or non-finite rows are encoded as the origin
-                        zx = __fmul_rn(__fmul_rn(x[m][2 * p], gn), q[m][p]);
-                        zy = __fmul_rn(__fmul_rn(x[m][2 * p + 1], gn), q[m][p]);
-                    }
-                    id[p] = uint32_t(a.brute ? search_exhaustive(s.cb, s.K, zx, zy) : search_table(s, zx, zy));
+                    float yx, yy;
+                    unpack2(mul2(P[rr][p], gn2), yx, yy);
+                    float zx = __fmul_rn(yx, q[rr][p]), zy = __fmul_rn(yy, q[rr][p]);
+                    if (!live) zx = zy = 0.f;
+                    id[p] = uint32_t(a.brute ? search_exhaustive(s, zx, zy) : search_table(s, zx, zy));
                 }
-                *reinterpret_cast<uint2*>(idx_s + k0) = make_uint2(id[0] | (id[1] << 16), id[2] | (id[3] << 16));
+                *reinterpret_cast<uint2*>(idx_s + stage_pos(k0)) = make_uint2(id[0] | (id[1] << 16), id[2] | (id[3] << 16));
             }
         }
         group_barrier(group, g.tg);
@@ -422,7 +601,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
             for (; k < n_pairs; ++k) {
                 const int sh = k * B - int(bit0);
                 if (sh >= 32) break;
-                const uint32_t v = idx_s[k];
+                const uint32_t v = idx_s[stage_pos(k)];
                 word |= sh >= 0 ? (v << sh) : (v >> (-sh));
             }
             out[w] = word;
@@ -446,7 +625,7 @@ struct AuxArgs {
     float* row_norm;
     // calibrate
     int n_calib_rows;        // rows visited: floor(t * d_out / n_calib_rows)
-    double* partial;         // [total_groups][n_pairs_padded] sums, then [total_groups] used-row counts
+    double* partial;         // [total_groups][pair_stride] sums, then [total_groups] used-row counts
     int pair_stride;
     int32_t* status;
 };
@@ -457,12 +636,15 @@ __global__ void __launch_bounds__(kMaxThreads, 1) aux_kernel(const AuxArgs a) {
     const RowGeom& g = a.g;
     const int group = threadIdx.x / g.tg;
     const int tid_g = threadIdx.x - group * g.tg;
-    const int lane_in_block = (LOG2B_T >= 5) ? (tid_g & ((1 << (LOG2B_T >= 5 ? LOG2B_T - 5 : 0)) - 1)) : 0;
     double* red = red_all + group * 64;
     const int n_pairs = g.d_in >> 1;
 
-    float t[4][8];
+    f32x2 t[4][4];
     load_col_factors<LOG2B_T>(t, a.chan_scale, a.signs, g.d_in, tid_g);
+    int e0s[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) e0s[r] = 8 * Layout<LOG2B_T>::octet_after(tid_g, r);
+    const bool y_vec = (g.d_in % 8 == 0) && (reinterpret_cast<uintptr_t>(a.y_out) % 16 == 0);
 
     const int n_rows = a.mode == 1 ? a.n_calib_rows : g.d_out;
     const long long total_groups = (long long)gridDim.x * g.groups;
@@ -474,63 +656,111 @@ __global__ void __launch_bounds__(kMaxThreads, 1) aux_kernel(const AuxArgs a) {
         for (int p = 0; p < 4; ++p) acc[m][p] = 0.0;
     int used = 0;
 
+    RawRow<BF16> raw;
+    if (my_group < n_rows) {
+        const long long row = a.mode == 1 ? (my_group * g.d_out) / a.n_calib_rows : my_group;
+        load_row<BF16, LOG2B_T>(raw, a.W, row, g, tid_g);
+    }
     int parity = 0;
     for (long long it = my_group; it < n_rows; it += total_groups, parity ^= 1) {
         const long long row = a.mode == 1 ? (it * g.d_out) / a.n_calib_rows : it;
-        RawRow<BF16> raw;
-        load_row<BF16, LOG2B_T>(raw, a.W, row, g, tid_g);
-        float x[4][8];
-        const float r = front_half<BF16, LOG2B_T>(raw, t, x, g, group, tid_g, lane_in_block, red, parity);
+        RawRow<BF16> nxt;
+        const long long it_next = it + total_groups;
+        if (it_next < n_rows) {
+            const long long row_next = a.mode == 1 ? (it_next * g.d_out) / a.n_calib_rows : it_next;
+            load_row<BF16, LOG2B_T>(nxt, a.W, row_next, g, tid_g);
+        }
+        f32x2 P[4][4];
+        const float r = front_half<BF16, LOG2B_T>(raw, t, P, g, group, tid_g, red, parity);
         const bool finite = isfinite(r);
         if (!finite && a.status && tid_g == 0) atomicOr(a.status, 1);
         const float gn = (finite && r > 0.f) ? inv_norm_factor(r, g.log2b) : 0.f;
+        const f32x2 gn2 = pack2(gn, gn);
         if (a.mode == 0) {
             if (tid_g == 0) a.row_norm[row] = r;
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                const int e0 = octet_offset<LOG2B_T>(tid_g, m);
+            for (int rr = 0; rr < 4; ++rr) {
+                if (e0s[rr] >= g.d_in) continue;
+                float y[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    if (e0 + e < g.d_in) a.y_out[row * g.d_in + e0 + e] = __fmul_rn(x[m][e], gn);
+                for (int i = 0; i < 4; ++i) unpack2(mul2(P[rr][i], gn2), y[2 * i], y[2 * i + 1]);
+                float* dst = a.y_out + row * g.d_in + e0s[rr];
+                if (y_vec) {
+                    reinterpret_cast<float4*>(dst)[0] = make_float4(y[0], y[1], y[2], y[3]);
+                    reinterpret_cast<float4*>(dst)[1] = make_float4(y[4], y[5], y[6], y[7]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if (e0s[rr] + e < g.d_in) dst[e] = y[e];
+                }
             }
         } else if (gn != 0.f) {
             ++used;
 #pragma unroll
-            for (int m = 0; m < 4; ++m)
+            for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
-                    const float y0 = __fmul_rn(x[m][2 * p], gn), y1 = __fmul_rn(x[m][2 * p + 1], gn);
-                    acc[m][p] += double(sqrtf(__fmaf_rn(y1, y1, __fmul_rn(y0, y0))));
+                    float y0, y1;
+                    unpack2(mul2(P[rr][p], gn2), y0, y1);
+                    acc[rr][p] += double(sqrtf(__fmaf_rn(y1, y1, __fmul_rn(y0, y0))));
                 }
         }
+        raw = nxt;
     }
     if (a.mode == 1) {
         double* mine = a.partial + my_group * a.pair_stride;
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            const int k0 = octet_offset<LOG2B_T>(tid_g, m) >> 1;
+        for (int rr = 0; rr < 4; ++rr) {
+            const int k0 = e0s[rr] >> 1;
 #pragma unroll
             for (int p = 0; p < 4; ++p)
-                if (k0 + p < n_pairs) mine[k0 + p] = acc[m][p];
+                if (k0 + p < n_pairs) mine[k0 + p] = acc[rr][p];
         }
         if (tid_g == 0) a.partial[total_groups * a.pair_stride + my_group] = double(used);
     }
 }
 
-// sigma_k from the per-group partial sums, added in group order (reproducible).
-__global__ void calibrate_finish_kernel(const double* partial, int total_groups, int pair_stride, int n_pairs,
-                                        int d_in, float* sigma_out) {
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= n_pairs) return;
-    double used = 0.0, sum = 0.0;
-    for (int gidx = 0; gidx < total_groups; ++gidx) {
-        used += partial[size_t(total_groups) * pair_stride + gidx];
-        sum += partial[size_t(gidx) * pair_stride + k];
+// sigma_k from the per-group partial sums.  A block owns 32 pair positions; its 8 warps each add
+// a contiguous slice of the groups in ascending order and the 8 slice sums are then added in
+// ascending order, so the result does not depend on timing.
+__global__ void __launch_bounds__(256) calibrate_finish_kernel(const double* partial, int total_groups, int pair_stride,
+                                                               int n_pairs, int d_in, float* sigma_out) {
+    __shared__ double part_sum[8][32], part_used[8];
+    const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
+    const int k = blockIdx.x * 32 + lane;
+    const int per = (total_groups + 7) / 8;
+    const int g0 = min(total_groups, slice * per), g1 = min(total_groups, g0 + per);
+    double sum = 0.0;
+    if (k < n_pairs) {
+        int gidx = g0;
+        for (; gidx + 4 <= g1; gidx += 4) {
+            const double v0 = partial[size_t(gidx) * pair_stride + k], v1 = partial[size_t(gidx + 1) * pair_stride + k];
+            const double v2 = partial[size_t(gidx + 2) * pair_stride + k], v3 = partial[size_t(gidx + 3) * pair_stride + k];
+            sum += v0;
+            sum += v1;
+            sum += v2;
+            sum += v3;
+        }
+        for (; gidx < g1; ++gidx) sum += partial[size_t(gidx) * pair_stride + k];
     }
-    const double inv_sqrt_d = 1.0 / sqrt(double(d_in));
-    double sg = used > 0.0 ? (sum / used) / sqrt(1.5707963267948966) : inv_sqrt_d;
-    sg = fmax(sg, 1e-4 * inv_sqrt_d);
-    sigma_out[k] = float(sg);
+    if (lane == 0) {
+        double used = 0.0;
+        for (int gidx = g0; gidx < g1; ++gidx) used += partial[size_t(total_groups) * pair_stride + gidx];
+        part_used[slice] = used;
+    }
+    part_sum[slice][lane] = sum;
+    __syncthreads();
+    if (slice == 0 && k < n_pairs) {
+        double s = 0.0, u = 0.0;
+        for (int i = 0; i < 8; ++i) {
+            s += part_sum[i][lane];
+            u += part_used[i];
+        }
+        const double inv_sqrt_d = 1.0 / sqrt(double(d_in));
+        double sg = u > 0.0 ? (s / u) / sqrt(1.5707963267948966) : inv_sqrt_d;
+        sg = fmax(sg, 1e-4 * inv_sqrt_d);
+        sigma_out[k] = float(sg);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -548,50 +778,59 @@ struct DecodeArgs {
     const float* sigma;
     const float2* codebook;  // device, K entries
     int K, log2K;
+    int log2c;               // log2 of the number of codebook copies in shared memory
     __nv_bfloat16* out;
 };
 
 template <int LOG2B_T>
 __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
-    float2* cb = reinterpret_cast<float2*>(smem);
-    for (int i = threadIdx.x; i < a.K; i += blockDim.x) cb[i] = a.codebook[i];
-    __syncthreads();
+    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
 
     const RowGeom& g = a.g;
     const int group = threadIdx.x / g.tg;
     const int tid_g = threadIdx.x - group * g.tg;
-    const int lane_in_block = (LOG2B_T >= 5) ? (tid_g & ((1 << (LOG2B_T >= 5 ? LOG2B_T - 5 : 0)) - 1)) : 0;
     const int n_pairs = g.d_in >> 1;
     const int B = a.log2K;
-    const uint32_t mask = (1u << B) - 1u;
+    const int cb_shift = 3 + a.log2c;
+    const uint32_t mask = ((1u << B) - 1u) << cb_shift;  // index mask, pre-shifted to a byte offset
+    const unsigned char* cb = smem + 8 * (threadIdx.x & ((1 << a.log2c) - 1));
 
-    // per-column output factor sign_j / (s_j sqrt(b)) and per-pair sigma
-    float mcol[4][8], sg[4][4];
+    // Input side: pair positions and pair scales of the octets in the slots before the rotation.
+    // Output side: element offsets and factors sign_j / (s_j sqrt(b)) of the slots after it.
+    int k_in[4], e_out[4];
+    float sg[4][4];
+    f32x2 mcol[4][4];
     const double inv_sqrt_b = 1.0 / sqrt(double(1 << g.log2b));
 #pragma unroll
-    for (int m = 0; m < 4; ++m) {
-        const int e0 = octet_offset<LOG2B_T>(tid_g, m);
+    for (int r = 0; r < 4; ++r) {
+        k_in[r] = 4 * Layout<LOG2B_T>::octet_before(tid_g, r);
+        e_out[r] = 8 * Layout<LOG2B_T>::octet_after(tid_g, r);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int j = e0 + e;
-            float v = 0.f;
-            if (j < g.d_in) v = float(double(a.signs[j]) * inv_sqrt_b / double(a.chan_scale ? a.chan_scale[j] : 1.0f));
-            mcol[m][e] = v;
+        for (int p = 0; p < 4; ++p) sg[r][p] = (k_in[r] + p < n_pairs) ? a.sigma[k_in[r] + p] : 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float v[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = e_out[r] + 2 * i + h;
+                v[h] = (j < g.d_in)
+                           ? float(double(a.signs[j]) * inv_sqrt_b / double(a.chan_scale ? a.chan_scale[j] : 1.0f))
+                           : 0.f;
+            }
+            mcol[r][i] = pack2(v[0], v[1]);
         }
-#pragma unroll
-        for (int p = 0; p < 4; ++p) sg[m][p] = ((e0 >> 1) + p < n_pairs) ? a.sigma[(e0 >> 1) + p] : 0.f;
     }
+    __syncthreads();
 
     const long long row_step = (long long)gridDim.x * g.groups;
     for (long long row = (long long)blockIdx.x * g.groups + group; row < g.d_out; row += row_step) {
         const uint32_t* in = reinterpret_cast<const uint32_t*>(a.packed + row * a.packed_row_stride);
-        const float r = a.row_norm[row];
-        float x[4][8];
+        const float rn = a.row_norm[row];
+        f32x2 P[4][4];
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            const int e0 = octet_offset<LOG2B_T>(tid_g, m);
-            const int k0 = e0 >> 1;
+        for (int r = 0; r < 4; ++r) {
+            const int k0 = k_in[r];
             if (k0 < n_pairs) {
                 const unsigned bit0 = unsigned(k0) * unsigned(B);
                 const int w0 = int(bit0 >> 5), sh = int(bit0 & 31u);
@@ -601,38 +840,40 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
                 // 64-bit window starting at bit `sh` of (hi:mid:lo); 4*B <= 48 bits are needed
                 unsigned long long win = ((unsigned long long)mid << 32 | lo) >> sh;
                 if (sh) win |= (unsigned long long)hi << (64 - sh);
+                win <<= cb_shift;  // indices become byte offsets into the lane's codebook copy (48 + 7 bits)
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
                     const bool valid = k0 + p < n_pairs;
-                    const uint32_t id = uint32_t(win >> (p * B)) & mask;
-                    const float2 c = cb[valid ? id : 0u];
-                    x[m][2 * p] = c.x * sg[m][p];
-                    x[m][2 * p + 1] = c.y * sg[m][p];
+                    const uint32_t off = uint32_t(win >> (p * B)) & mask;
+                    const float2 c = *reinterpret_cast<const float2*>(cb + (valid ? off : 0u));
+                    P[r][p] = pack2(c.x * sg[r][p], c.y * sg[r][p]);
                 }
             } else {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) x[m][e] = 0.f;
+                for (int p = 0; p < 4; ++p) P[r][p] = pack2(0.f, 0.f);
             }
         }
-        fwht_regs<LOG2B_T>(x, g.log2b, lane_in_block);
+        fwht_regs<LOG2B_T>(P, g.log2b, tid_g);
+        const f32x2 rn2 = pack2(rn, rn);
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            const int e0 = octet_offset<LOG2B_T>(tid_g, m);
+        for (int r = 0; r < 4; ++r) {
+            const int e0 = e_out[r];
             if (e0 >= g.d_in) continue;
             __nv_bfloat16* dst = a.out + row * g.d_in + e0;
-            if (g.vec) {
-                uint32_t w[4];
+            uint32_t w[4];
+            float y[8];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    __nv_bfloat162 h2 = __floats2bfloat162_rn(x[m][2 * i] * (mcol[m][2 * i] * r),
-                                                              x[m][2 * i + 1] * (mcol[m][2 * i + 1] * r));
-                    w[i] = *reinterpret_cast<uint32_t*>(&h2);
-                }
+            for (int i = 0; i < 4; ++i) {
+                unpack2(mul2(P[r][i], mul2(mcol[r][i], rn2)), y[2 * i], y[2 * i + 1]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
+                w[i] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            if (g.vec) {
                 *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
             } else {
 #pragma unroll
                 for (int e = 0; e < 8; ++e)
-                    if (e0 + e < g.d_in) dst[e] = __float2bfloat16_rn(x[m][e] * (mcol[m][e] * r));
+                    if (e0 + e < g.d_in) dst[e] = __float2bfloat16_rn(y[e]);
             }
         }
     }
@@ -642,32 +883,112 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
 // distortion kernel
 // ---------------------------------------------------------------------------------------------
 
+// A block walks over (row chunk, column tile) work items; a thread owns 8 consecutive columns of
+// the tile and accumulates, per column, sum e^2 and sum w^2 over the rows of the chunk in double;
+// the activation weights r_j^2 are applied once per column at the end of the chunk.
+constexpr int kDistThreads = 128;
+constexpr int kDistRows = 32;
+
 template <bool BF16>
-__global__ void __launch_bounds__(256) distortion_kernel(const void* W, long long w_row_stride, const __nv_bfloat16* What,
-                                                         const float* act_rms, int d_out, int d_in, double* out4) {
-    double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
-    for (long long row = blockIdx.x; row < d_out; row += gridDim.x) {
-        const char* wrow = static_cast<const char*>(W) + row * w_row_stride * (BF16 ? 2 : 4);
-        const __nv_bfloat16* hrow = What + row * d_in;
-        for (int j = threadIdx.x; j < d_in; j += blockDim.x) {
-            const float w = BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(wrow)[j])
-                                 : reinterpret_cast<const float*>(wrow)[j];
-            const double wd = double(w), e = wd - double(__bfloat162float(hrow[j]));
-            const double r2 = act_rms ? double(act_rms[j]) * double(act_rms[j]) : 1.0;
-            s0 += e * e;
-            s1 += wd * wd;
-            s2 += r2 * e * e;
-            s3 += r2 * wd * wd;
+__device__ __forceinline__ void dist_load(const void* W, long long w_row_stride, const __nv_bfloat16* What, int row,
+                                          int j0, int d_in, int vec, float (&w)[8], float (&h)[8]) {
+    const char* wrow = static_cast<const char*>(W) + (long long)row * w_row_stride * (BF16 ? 2 : 4);
+    const __nv_bfloat16* hrow = What + (long long)row * d_in;
+    if (vec) {
+        const uint4 hv = __ldg(reinterpret_cast<const uint4*>(hrow + j0));
+        const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            h[2 * i] = __uint_as_float(hw[i] << 16);
+            h[2 * i + 1] = __uint_as_float(hw[i] & 0xffff0000u);
+        }
+        if (BF16) {
+            const uint4 wv = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(wrow) + j0));
+            const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                w[2 * i] = __uint_as_float(ww[i] << 16);
+                w[2 * i + 1] = __uint_as_float(ww[i] & 0xffff0000u);
+            }
+        } else {
+            const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(wrow) + j0);
+            const float4 a = __ldg(p), c = __ldg(p + 1);
+            w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
+            w[4] = c.x; w[5] = c.y; w[6] = c.z; w[7] = c.w;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const bool in = j0 + e < d_in;
+            h[e] = in ? __bfloat162float(hrow[j0 + e]) : 0.f;
+            w[e] = !in ? 0.f
+                       : (BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(wrow)[j0 + e])
+                               : reinterpret_cast<const float*>(wrow)[j0 + e]);
         }
     }
-    __shared__ double sh[4][8];
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kDistThreads) distortion_kernel(const void* W, long long w_row_stride,
+                                                                  const __nv_bfloat16* What, const float* act_rms,
+                                                                  int d_out, int d_in, int vec, double* out4) {
+    const int col_tiles = (d_in + 8 * kDistThreads - 1) / (8 * kDistThreads);
+    const int row_chunks = (d_out + kDistRows - 1) / kDistRows;
+    const long long n_items = (long long)col_tiles * row_chunks;
+    double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int chunk = int(item / col_tiles), tile = int(item - (long long)chunk * col_tiles);
+        const int j0 = (tile * kDistThreads + threadIdx.x) * 8;
+        if (j0 >= d_in) continue;
+        const int r0 = chunk * kDistRows, r1 = min(d_out, r0 + kDistRows);
+        double E[8], Q[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) E[e] = Q[e] = 0.0;
+        int row = r0;
+        for (; row + 4 <= r1; row += 4) {  // four rows in flight
+            float w[4][8], h[4][8];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) dist_load<BF16>(W, w_row_stride, What, row + u, j0, d_in, vec, w[u], h[u]);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const double wd = double(w[u][e]), d = wd - double(h[u][e]);
+                    E[e] = fma(d, d, E[e]);
+                    Q[e] = fma(wd, wd, Q[e]);
+                }
+        }
+        for (; row < r1; ++row) {
+            float w[8], h[8];
+            dist_load<BF16>(W, w_row_stride, What, row, j0, d_in, vec, w, h);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const double wd = double(w[e]), d = wd - double(h[e]);
+                E[e] = fma(d, d, E[e]);
+                Q[e] = fma(wd, wd, Q[e]);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            double r2 = 1.0;
+            if (act_rms && j0 + e < d_in) {
+                const double rj = double(act_rms[j0 + e]);
+                r2 = rj * rj;
+            }
+            s0 += E[e];
+            s1 += Q[e];
+            s2 = fma(r2, E[e], s2);
+            s3 = fma(r2, Q[e], s3);
+        }
+    }
+    __shared__ double sh[4][kDistThreads / 32];
     s0 = warp_sum(s0); s1 = warp_sum(s1); s2 = warp_sum(s2); s3 = warp_sum(s3);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (lane == 0) { sh[0][warp] = s0; sh[1][warp] = s1; sh[2][warp] = s2; sh[3][warp] = s3; }
     __syncthreads();
     if (threadIdx.x < 4) {
         double v = 0;
-        for (int w = 0; w < int(blockDim.x >> 5); ++w) v += sh[threadIdx.x][w];
+        for (int w = 0; w < kDistThreads / 32; ++w) v += sh[threadIdx.x][w];
         atomicAdd(out4 + threadIdx.x, v);
     }
 }
@@ -735,6 +1056,14 @@ int set_smem(Kernel k, size_t bytes) {
     return QAMW_OK;
 }
 
+// Largest power-of-two number of codebook copies (at most 16: one per 8-byte bank pair) that
+// fits into `budget` bytes of shared memory.
+int pick_log2_copies(int K, size_t budget) {
+    int log2c = 4;
+    while (log2c > 0 && (size_t(K) * 8 << log2c) > budget) --log2c;
+    return log2c;
+}
+
 template <bool BF16, int LOG2B_T>
 int launch_encode(const EncodeArgs& a, int blocks, size_t smem, cudaStream_t st) {
     int rc = set_smem(encode_kernel<BF16, LOG2B_T>, smem);
@@ -782,8 +1111,10 @@ extern "C" int qamw_codebook_create(const float* codebook_host, int K, int grid,
     if (grid < 0 || grid > 255) return QAMW_ERR_ARG;
     *out = nullptr;
     SearchTable t;
-    // leave room for the per-group scratch of the encoder inside the 227 KB of one SM
-    const size_t budget = size_t(200) * 1024 - size_t(K) * 8;
+    // The encoder's shared memory also holds several codebook copies (at least 64 KB worth, two
+    // copies for K = 4096) and about 24 KB of per-group scratch: the table gets what is left of
+    // the 227 KB of one SM.
+    const size_t budget = size_t(227 - 24) * 1024 - std::max(size_t(64) * 1024, size_t(K) * 16);
     if (!choose_search_table(codebook_host, K, grid, budget, &t)) return QAMW_ERR_NOMEM;
     qamw_codebook* cb = new (std::nothrow) qamw_codebook();
     if (!cb) return QAMW_ERR_NOMEM;
@@ -849,11 +1180,11 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     a.chan_scale = chan_scale;
     a.signs = signs;
     a.sigma = sigma;
-    a.blob = static_cast<const uint4*>(cb->d_blob);
-    a.blob_bytes = int(cb->blob_bytes);
-    a.off_cells = int(cb->off_cells);
-    a.off_overflow = int(cb->off_overflow);
-    a.off_lut = int(cb->off_lut);
+    a.codebook = static_cast<const float2*>(cb->d_blob);
+    a.table = reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(cb->d_blob) + cb->off_cells);
+    a.table_bytes = int(cb->blob_bytes - cb->off_cells);
+    a.off_overflow = int(cb->off_overflow - cb->off_cells);
+    a.off_lut = int(cb->off_lut - cb->off_cells);
     a.K = p->K;
     a.log2K = ilog2(p->K);
     a.grid = cb->grid;
@@ -863,10 +1194,13 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     a.row_words = int(p->packed_row_stride / 4);
     a.row_norm = row_norm_out;
     a.status = status_out;
-    a.idx_stride = ((p->d_in / 2 + 7) / 8) * 8 + 8;
-    const size_t smem = ((cb->blob_bytes + 15) & ~size_t(15)) + size_t(a.g.groups) * 64 * sizeof(double) +
-                        size_t(a.g.groups) * a.idx_stride * 2;
-    if (smem > 227 * 1024) return QAMW_ERR_NOMEM;
+    const int n_pairs = p->d_in / 2;
+    a.idx_stride = ((n_pairs + (n_pairs >> 6) * 16 + 7) / 8) * 8 + 24;
+    const size_t fixed = ((size_t(a.table_bytes) + 15) & ~size_t(15)) + size_t(a.g.groups) * 64 * sizeof(double) +
+                         size_t(a.g.groups) * a.idx_stride * 2;
+    if (fixed + size_t(p->K) * 8 > kSmemLimit) return QAMW_ERR_NOMEM;
+    a.log2c = pick_log2_copies(p->K, kSmemLimit - fixed);
+    const size_t smem = fixed + (size_t(p->K) * 8 << a.log2c);
     const int blocks = std::max(1, std::min(sm_count(), (p->d_out + a.g.groups - 1) / a.g.groups));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define CALL(LB)                                                                  \
@@ -946,8 +1280,8 @@ extern "C" int qamw_calibrate(const void* W, const qamw_params* p, const float* 
 #undef CALL
     if (rc) return rc;
     const int n_pairs = p->d_in / 2;
-    calibrate_finish_kernel<<<(n_pairs + 127) / 128, 128, 0, st>>>(a.partial, c.total_groups, c.pair_stride, n_pairs,
-                                                                    p->d_in, sigma_out);
+    calibrate_finish_kernel<<<(n_pairs + 31) / 32, 256, 0, st>>>(a.partial, c.total_groups, c.pair_stride, n_pairs,
+                                                                  p->d_in, sigma_out);
     return finish_launch("calibrate_finish_kernel");
 }
 
@@ -1028,8 +1362,9 @@ extern "C" int qamw_decode(const uint8_t* packed, const float* row_norm, const f
     a.codebook = static_cast<const float2*>(cb->d_blob);
     a.K = p->K;
     a.log2K = ilog2(p->K);
+    a.log2c = pick_log2_copies(p->K, size_t(128) * 1024);
     a.out = static_cast<__nv_bfloat16*>(w_hat_bf16_out);
-    const size_t smem = size_t(p->K) * 8;
+    const size_t smem = size_t(p->K) * 8 << a.log2c;
     const int blocks = std::max(1, std::min(sm_count(), (p->d_out + a.g.groups - 1) / a.g.groups));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define CALL(LB) rc = launch_decode<LB>(a, blocks, smem, st)
@@ -1050,12 +1385,19 @@ extern "C" int qamw_distortion(const void* W, const void* w_hat_bf16, const floa
         return QAMW_ERR_CUDA;
     }
     if (p->d_out == 0) return QAMW_OK;
-    const int blocks = std::max(1, std::min(4 * sm_count(), p->d_out));
+    const size_t esz = p->w_dtype == QAMW_DTYPE_BF16 ? 2 : 4;
+    const int vec = (p->d_in % 8 == 0) && (reinterpret_cast<uintptr_t>(W) % 16 == 0) &&
+                    ((size_t(p->w_row_stride) * esz) % 16 == 0) && (reinterpret_cast<uintptr_t>(w_hat_bf16) % 16 == 0);
+    const long long items = (long long)((p->d_in + 8 * kDistThreads - 1) / (8 * kDistThreads)) *
+                            ((p->d_out + kDistRows - 1) / kDistRows);
+    const int blocks = int(std::max<long long>(1, std::min<long long>(16LL * sm_count(), items)));
     if (p->w_dtype == QAMW_DTYPE_BF16)
-        distortion_kernel<true><<<blocks, 256, 0, st>>>(W, p->w_row_stride, static_cast<const __nv_bfloat16*>(w_hat_bf16),
-                                                        act_rms, p->d_out, p->d_in, out4);
+        distortion_kernel<true><<<blocks, kDistThreads, 0, st>>>(W, p->w_row_stride,
+                                                                 static_cast<const __nv_bfloat16*>(w_hat_bf16), act_rms,
+                                                                 p->d_out, p->d_in, vec, out4);
     else
-        distortion_kernel<false><<<blocks, 256, 0, st>>>(W, p->w_row_stride, static_cast<const __nv_bfloat16*>(w_hat_bf16),
-                                                         act_rms, p->d_out, p->d_in, out4);
+        distortion_kernel<false><<<blocks, kDistThreads, 0, st>>>(W, p->w_row_stride,
+                                                                  static_cast<const __nv_bfloat16*>(w_hat_bf16), act_rms,
+                                                                  p->d_out, p->d_in, vec, out4);
     return finish_launch("distortion_kernel");
 }
