@@ -398,8 +398,29 @@ __device__ __forceinline__ float inv_norm_factor(float r, int log2b) {
 // (lane mod C) only ever touches its own 16/C bank pairs.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void fill_codebook_copies(float2* dst, const float2* src, int K, int log2c) {
-    const int n = K << log2c;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) dst[i] = __ldg(src + (i >> log2c));
+    // all loads of a thread first (up to 8 in flight), then the copies as 16-byte stores
+    constexpr int kMaxPerThread = 8;
+    float2 c[kMaxPerThread];
+    const int T = blockDim.x;
+    for (int base = 0; base < K; base += kMaxPerThread * T) {
+#pragma unroll
+        for (int u = 0; u < kMaxPerThread; ++u) {
+            const int i = base + u * T + threadIdx.x;
+            c[u] = i < K ? __ldg(src + i) : make_float2(0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < kMaxPerThread; ++u) {
+            const int i = base + u * T + threadIdx.x;
+            if (i >= K) continue;
+            if (log2c == 0) {
+                dst[i] = c[u];
+            } else {
+                float4* d4 = reinterpret_cast<float4*>(dst + (size_t(i) << log2c));
+                const float4 v = make_float4(c[u].x, c[u].y, c[u].x, c[u].y);
+                for (int k = 0; k < (1 << (log2c - 1)); ++k) d4[k] = v;
+            }
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -771,7 +792,11 @@ struct DecodeArgs {
     RowGeom g;               // d_out, d_in, log2b, tg, groups; vec = output rows 16-byte aligned
     const uint8_t* packed;
     long long packed_row_stride;
-    int row_words;           // readable 32-bit words per packed row
+    int row_bytes;           // bytes of a packed row that may be copied (payload rounded up to the copy size)
+    int copy_log2;           // log2 of the async copy size: 4 when rows are 16-byte aligned, else 2
+    int seg_bytes;           // packed bytes of the 512 pairs of one warp: 64 * B
+    int stage_bytes;         // one staging buffer of a warp: seg_bytes + 16
+    float inv_sqrt_b;        // f32(1 / sqrt(b))
     const float* row_norm;
     const float* chan_scale;
     const int8_t* signs;
@@ -782,70 +807,106 @@ struct DecodeArgs {
     __nv_bfloat16* out;
 };
 
+// Asynchronous global -> shared copies (no register staging, completion tracked per thread).
+__device__ __forceinline__ void cp_async(void* smem_dst, const void* gmem_src, int log2_bytes) {
+    const unsigned dst = unsigned(__cvta_generic_to_shared(smem_dst));
+    if (log2_bytes == 4)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+    else
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// A warp owns 1024 consecutive elements of its row, i.e. 512 pairs = 64*B consecutive bytes of the
+// packed row (a multiple of 16 for every B).  Each warp streams that segment through its own
+// two-deep shared-memory ring: while a row is decoded the next one is on its way, and since
+// nothing is shared between warps the kernel has no barrier after its prologue.
 template <int LOG2B_T>
 __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
-    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
-
     const RowGeom& g = a.g;
     const int group = threadIdx.x / g.tg;
     const int tid_g = threadIdx.x - group * g.tg;
+    const int lane = threadIdx.x & 31;
     const int n_pairs = g.d_in >> 1;
     const int B = a.log2K;
-    const int cb_shift = 3 + a.log2c;
-    const uint32_t mask = ((1u << B) - 1u) << cb_shift;  // index mask, pre-shifted to a byte offset
+    const uint32_t mask = (1u << B) - 1u;
+    const uint32_t cb_stride = 8u << a.log2c;
     const unsigned char* cb = smem + 8 * (threadIdx.x & ((1 << a.log2c) - 1));
+    unsigned char* stage = smem + ((size_t(a.K) * 8) << a.log2c) + size_t(threadIdx.x >> 5) * 2 * a.stage_bytes;
 
-    // Input side: pair positions and pair scales of the octets in the slots before the rotation.
+    // first row on its way before anything else
+    const long long seg_off = (long long)(tid_g >> 5) * a.seg_bytes;  // of this warp's segment inside a packed row
+    const int seg_len = int(max(0LL, min((long long)a.seg_bytes, (long long)a.row_bytes - seg_off)));
+    const int n_chunks = seg_len >> a.copy_log2;
+    auto issue_row = [&](long long row, int buf) {
+        const unsigned char* src = a.packed + row * a.packed_row_stride + seg_off;
+        unsigned char* dst = stage + buf * a.stage_bytes;
+        for (int c = lane; c < n_chunks; c += 32)
+            cp_async(dst + (size_t(c) << a.copy_log2), src + (size_t(c) << a.copy_log2), a.copy_log2);
+        cp_async_commit();
+    };
+    const long long row_step = (long long)gridDim.x * g.groups;
+    long long row = (long long)blockIdx.x * g.groups + group;
+    if (row < g.d_out) issue_row(row, 0);
+    // the 16 bytes after a staged segment are read (and masked away) by the last windows: keep them defined
+    if (lane < 8) reinterpret_cast<uint32_t*>(stage + (lane >> 2) * a.stage_bytes + a.seg_bytes)[lane & 3] = 0u;
+
+    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
+
+    // Input side: window position and pair scales of the octets in the slots before the rotation.
     // Output side: element offsets and factors sign_j / (s_j sqrt(b)) of the slots after it.
-    int k_in[4], e_out[4];
+    int e_out[4], w0s[4], shs[4];
+    bool live[4];
     float sg[4][4];
     f32x2 mcol[4][4];
-    const double inv_sqrt_b = 1.0 / sqrt(double(1 << g.log2b));
+    const int warp_pair0 = (tid_g & ~31) * 16;  // first pair of this warp's segment
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-        k_in[r] = 4 * Layout<LOG2B_T>::octet_before(tid_g, r);
+        const int k0 = 4 * Layout<LOG2B_T>::octet_before(tid_g, r);
+        live[r] = k0 < n_pairs;
+        const unsigned bit0 = unsigned(k0 - warp_pair0) * unsigned(B);
+        w0s[r] = int(bit0 >> 5);
+        shs[r] = int(bit0 & 31u);
         e_out[r] = 8 * Layout<LOG2B_T>::octet_after(tid_g, r);
 #pragma unroll
-        for (int p = 0; p < 4; ++p) sg[r][p] = (k_in[r] + p < n_pairs) ? a.sigma[k_in[r] + p] : 0.f;
+        for (int p = 0; p < 4; ++p) sg[r][p] = (k0 + p < n_pairs) ? a.sigma[k0 + p] : 0.f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             float v[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int j = e_out[r] + 2 * i + h;
-                v[h] = (j < g.d_in)
-                           ? float(double(a.signs[j]) * inv_sqrt_b / double(a.chan_scale ? a.chan_scale[j] : 1.0f))
-                           : 0.f;
+                v[h] = (j < g.d_in) ? __fdiv_rn(float(a.signs[j]) * a.inv_sqrt_b, a.chan_scale ? a.chan_scale[j] : 1.0f) : 0.f;
             }
             mcol[r][i] = pack2(v[0], v[1]);
         }
     }
     __syncthreads();
 
-    const long long row_step = (long long)gridDim.x * g.groups;
-    for (long long row = (long long)blockIdx.x * g.groups + group; row < g.d_out; row += row_step) {
-        const uint32_t* in = reinterpret_cast<const uint32_t*>(a.packed + row * a.packed_row_stride);
+    int buf = 0;
+    for (; row < g.d_out; row += row_step, buf ^= 1) {
         const float rn = a.row_norm[row];
+        cp_async_wait_all();
+        __syncwarp();  // every lane's part of this row has landed; the other buffer is no longer read
+        if (row + row_step < g.d_out) issue_row(row + row_step, buf ^ 1);
+        const uint32_t* in = reinterpret_cast<const uint32_t*>(stage + buf * a.stage_bytes);
         f32x2 P[4][4];
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-            const int k0 = k_in[r];
-            if (k0 < n_pairs) {
-                const unsigned bit0 = unsigned(k0) * unsigned(B);
-                const int w0 = int(bit0 >> 5), sh = int(bit0 & 31u);
-                const uint32_t lo = __ldg(in + w0);
-                const uint32_t mid = (w0 + 1 < a.row_words) ? __ldg(in + w0 + 1) : 0u;
-                const uint32_t hi = (w0 + 2 < a.row_words) ? __ldg(in + w0 + 2) : 0u;
-                // 64-bit window starting at bit `sh` of (hi:mid:lo); 4*B <= 48 bits are needed
-                unsigned long long win = ((unsigned long long)mid << 32 | lo) >> sh;
-                if (sh) win |= (unsigned long long)hi << (64 - sh);
-                win <<= cb_shift;  // indices become byte offsets into the lane's codebook copy (48 + 7 bits)
+            if (live[r]) {
+                const uint32_t* w = in + w0s[r];
+                const uint32_t lo = w[0], mid = w[1], hi = w[2];
+                // bits [sh, sh+64) of (hi:mid:lo) as two words; pairs 0,1 come from the first word,
+                // pairs 2,3 from the 32 bits that start 2B further on (4B <= 48)
+                const uint32_t a0 = __funnelshift_r(lo, mid, shs[r]), a1 = __funnelshift_r(mid, hi, shs[r]);
+                const uint32_t b0 = __funnelshift_r(a0, a1, 2 * B);
+                const uint32_t id[4] = {a0 & mask, (a0 >> B) & mask, b0 & mask, (b0 >> B) & mask};
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
-                    const bool valid = k0 + p < n_pairs;
-                    const uint32_t off = uint32_t(win >> (p * B)) & mask;
-                    const float2 c = *reinterpret_cast<const float2*>(cb + (valid ? off : 0u));
+                    // pairs past the end of a row whose length is not a multiple of 8 have scale 0
+                    const float2 c = *reinterpret_cast<const float2*>(cb + id[p] * cb_stride);
                     P[r][p] = pack2(c.x * sg[r][p], c.y * sg[r][p]);
                 }
             } else {
@@ -1354,17 +1415,24 @@ extern "C" int qamw_decode(const uint8_t* packed, const float* row_norm, const f
     a.g.vec = (p->d_in % 8 == 0) && (reinterpret_cast<uintptr_t>(w_hat_bf16_out) % 16 == 0);
     a.packed = packed;
     a.packed_row_stride = p->packed_row_stride;
-    a.row_words = int(p->packed_row_stride / 4);
+    a.row_bytes = int((row_bytes + 3) / 4 * 4);
+    const bool rows16 = reinterpret_cast<uintptr_t>(packed) % 16 == 0 && p->packed_row_stride % 16 == 0;
+    a.copy_log2 = rows16 ? 4 : 2;
+    if (rows16) a.row_bytes = int((row_bytes + 15) / 16 * 16);  // <= the stride, which is a multiple of 16
+    a.log2K = ilog2(p->K);
+    a.seg_bytes = 64 * a.log2K;
+    a.stage_bytes = a.seg_bytes + 16;
+    a.inv_sqrt_b = float(1.0 / std::sqrt(double(p->block)));
     a.row_norm = row_norm;
     a.chan_scale = chan_scale;
     a.signs = signs;
     a.sigma = sigma;
     a.codebook = static_cast<const float2*>(cb->d_blob);
     a.K = p->K;
-    a.log2K = ilog2(p->K);
-    a.log2c = pick_log2_copies(p->K, size_t(128) * 1024);
     a.out = static_cast<__nv_bfloat16*>(w_hat_bf16_out);
-    const size_t smem = size_t(p->K) * 8 << a.log2c;
+    const size_t stage_total = size_t(a.g.groups) * (a.g.tg / 32) * 2 * a.stage_bytes;
+    a.log2c = pick_log2_copies(p->K, std::min(size_t(128) * 1024, kSmemLimit - stage_total));
+    const size_t smem = (size_t(p->K) * 8 << a.log2c) + stage_total;
     const int blocks = std::max(1, std::min(sm_count(), (p->d_out + a.g.groups - 1) / a.g.groups));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define CALL(LB) rc = launch_decode<LB>(a, blocks, smem, st)
