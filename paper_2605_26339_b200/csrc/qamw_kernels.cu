@@ -58,6 +58,7 @@ struct RowGeom {
     int tg;           // threads per group (multiple of 32)
     int groups;       // groups per thread block
     int vec;          // rows can be moved with 16-byte accesses
+    int cvec;         // per-column constants (channel scales, signs, sigma) can be read with vector loads
     int w_bf16;       // 1 = bf16 weights, 0 = f32
     long long w_row_stride;  // elements
 };
@@ -334,25 +335,71 @@ __device__ __forceinline__ void raw_to_float(const RawRow<BF16>& raw, float (&x)
     }
 }
 
-// Per-thread column constants of the encoder side: t_j = f32(s_j) * sign_j (0 beyond the row),
-// for the columns the thread holds when the row is loaded.
+// Eight consecutive per-column constants starting at column e0 (a multiple of 8): 16-byte loads
+// when the arrays allow it (checked on the host: `cvec`), element-wise otherwise.  Columns beyond
+// n read as `fill`.
+__device__ __forceinline__ void load8f(const float* p, int e0, int n, int cvec, float fill, float (&v)[8]) {
+    if (cvec && e0 + 8 <= n) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(p + e0));
+        const float4 c = __ldg(reinterpret_cast<const float4*>(p + e0) + 1);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+        v[4] = c.x; v[5] = c.y; v[6] = c.z; v[7] = c.w;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = (e0 + e < n) ? __ldg(p + e0 + e) : fill;
+    }
+}
+__device__ __forceinline__ void load4f(const float* p, int k0, int n, int cvec, float fill, float (&v)[4]) {
+    if (cvec && k0 + 4 <= n) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(p + k0));
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = (k0 + e < n) ? __ldg(p + k0 + e) : fill;
+    }
+}
+// signs (+1 / -1 bytes) of 8 consecutive columns as floats; 0 beyond n
+__device__ __forceinline__ void load8s(const int8_t* p, int e0, int n, int cvec, float (&v)[8]) {
+    if (cvec && e0 + 8 <= n) {
+        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(p + e0));
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const uint32_t w = e < 4 ? raw.x : raw.y;
+            const uint32_t byte = (w >> (8 * (e & 3))) & 0xffu;
+            v[e] = __uint_as_float(0x3f800000u | ((byte & 0x80u) << 24));  // +-1.0f from the byte's sign bit
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = (e0 + e < n) ? float(__ldg(p + e0 + e)) : 0.f;
+    }
+}
+
+// Raw per-column inputs of the encoder side for the octets a thread holds when the row is loaded.
+struct ColRaw {
+    float cs[4][8];   // channel scales (1 when there are none)
+    float sgn[4][8];  // signs, 0 beyond the row
+};
 template <int LOG2B_T>
-__device__ __forceinline__ void load_col_factors(f32x2 (&t)[4][4], const float* chan_scale, const int8_t* signs,
-                                                 int d_in, int tid_g) {
+__device__ __forceinline__ void load_col_raw(ColRaw& c, const float* chan_scale, const int8_t* signs, int d_in,
+                                             int cvec, int tid_g) {
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
         const int e0 = 8 * Layout<LOG2B_T>::octet_before(tid_g, r);
+        if (chan_scale) {
+            load8f(chan_scale, e0, d_in, cvec, 1.0f, c.cs[r]);
+        } else {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float v[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int j = e0 + 2 * i + h;
-                v[h] = (j < d_in) ? (chan_scale ? chan_scale[j] : 1.0f) * float(signs[j]) : 0.f;
-            }
-            t[r][i] = pack2(v[0], v[1]);
+            for (int e = 0; e < 8; ++e) c.cs[r][e] = 1.0f;
         }
+        load8s(signs, e0, d_in, cvec, c.sgn[r]);
     }
+}
+// t_j = f32(s_j) * sign_j (0 beyond the row)
+__device__ __forceinline__ void col_factors(const ColRaw& c, f32x2 (&t)[4][4]) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) t[r][i] = pack2(c.cs[r][2 * i] * c.sgn[r][2 * i], c.cs[r][2 * i + 1] * c.sgn[r][2 * i + 1]);
 }
 
 // Scaling, row norm and butterfly of one row held in registers (the arithmetic contract of the
@@ -532,16 +579,51 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     extern __shared__ __align__(16) unsigned char smem[];
     const RowGeom& g = a.g;
     // shared memory: [codebook copies][table][red: groups x 64 doubles][idx: groups x idx_stride u16]
+    const int group = threadIdx.x / g.tg;
+    const int tid_g = threadIdx.x - group * g.tg;
+    const int n_pairs = g.d_in >> 1;
+    // all global loads of the prologue are issued before anything waits for one of them
+    ColRaw craw;
+    load_col_raw<LOG2B_T>(craw, a.chan_scale, a.signs, g.d_in, g.cvec, tid_g);
+    int k0s[4];
+    float q[4][4];  // pair positions and reciprocal pair scales of the octets held after the rotation
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        k0s[r] = 4 * Layout<LOG2B_T>::octet_after(tid_g, r);
+        load4f(a.sigma, k0s[r], n_pairs, g.cvec, 1.0f, q[r]);
+    }
     const int cb_bytes = (a.K * 8) << a.log2c;
     fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
     unsigned char* table = smem + cb_bytes;
     {
         uint4* dst = reinterpret_cast<uint4*>(table);
-        for (int i = threadIdx.x; i < a.table_bytes / 16; i += blockDim.x) dst[i] = __ldg(a.table + i);
+        const int n16 = a.table_bytes / 16;
+        for (int base = 0; base < n16; base += 8 * blockDim.x) {
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = base + u * blockDim.x + threadIdx.x;
+                if (i < n16) v[u] = __ldg(a.table + i);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = base + u * blockDim.x + threadIdx.x;
+                if (i < n16) dst[i] = v[u];
+            }
+        }
     }
     const int table_pad = (a.table_bytes + 15) & ~15;
     double* red_all = reinterpret_cast<double*>(table + table_pad);
     uint16_t* idx_all = reinterpret_cast<uint16_t*>(table + table_pad + g.groups * 64 * sizeof(double));
+
+    f32x2 t[4][4];
+    col_factors(craw, t);
+    // q_k = f32(1 / (double)sigma_k): the correctly rounded f32 reciprocal is the same number (the
+    // exact quotient of two f32 is never within 2^-53 of an f32 rounding boundary unless it is exact)
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int p = 0; p < 4; ++p) q[r][p] = (k0s[r] + p < n_pairs) ? __frcp_rn(q[r][p]) : 0.f;
     __syncthreads();
 
     SearchSmem s;
@@ -553,23 +635,8 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     s.grid = a.grid;
     s.K = a.K;
 
-    const int group = threadIdx.x / g.tg;
-    const int tid_g = threadIdx.x - group * g.tg;
     double* red = red_all + group * 64;
     uint16_t* idx_s = idx_all + size_t(group) * a.idx_stride;
-    const int n_pairs = g.d_in >> 1;
-
-    f32x2 t[4][4];
-    load_col_factors<LOG2B_T>(t, a.chan_scale, a.signs, g.d_in, tid_g);
-    // pair positions and reciprocal pair scales of the octets the thread holds after the rotation
-    int k0s[4];
-    float q[4][4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        k0s[r] = 4 * Layout<LOG2B_T>::octet_after(tid_g, r);
-#pragma unroll
-        for (int p = 0; p < 4; ++p) q[r][p] = (k0s[r] + p < n_pairs) ? float(1.0 / double(a.sigma[k0s[r] + p])) : 0.f;
-    }
 
     const long long row_step = (long long)gridDim.x * g.groups;
     long long row = (long long)blockIdx.x * g.groups + group;
@@ -661,7 +728,11 @@ __global__ void __launch_bounds__(kMaxThreads, 1) aux_kernel(const AuxArgs a) {
     const int n_pairs = g.d_in >> 1;
 
     f32x2 t[4][4];
-    load_col_factors<LOG2B_T>(t, a.chan_scale, a.signs, g.d_in, tid_g);
+    {
+        ColRaw craw;
+        load_col_raw<LOG2B_T>(craw, a.chan_scale, a.signs, g.d_in, g.cvec, tid_g);
+        col_factors(craw, t);
+    }
     int e0s[4];
 #pragma unroll
     for (int r = 0; r < 4; ++r) e0s[r] = 8 * Layout<LOG2B_T>::octet_after(tid_g, r);
@@ -853,14 +924,13 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
     // the 16 bytes after a staged segment are read (and masked away) by the last windows: keep them defined
     if (lane < 8) reinterpret_cast<uint32_t*>(stage + (lane >> 2) * a.stage_bytes + a.seg_bytes)[lane & 3] = 0u;
 
-    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
-
     // Input side: window position and pair scales of the octets in the slots before the rotation.
     // Output side: element offsets and factors sign_j / (s_j sqrt(b)) of the slots after it.
+    // The global loads of these constants and of the codebook are all issued before the first use.
     int e_out[4], w0s[4], shs[4];
     bool live[4];
     float sg[4][4];
-    f32x2 mcol[4][4];
+    float cs[4][8], sgn[4][8];
     const int warp_pair0 = (tid_g & ~31) * 16;  // first pair of this warp's segment
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
@@ -870,19 +940,23 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
         w0s[r] = int(bit0 >> 5);
         shs[r] = int(bit0 & 31u);
         e_out[r] = 8 * Layout<LOG2B_T>::octet_after(tid_g, r);
+        load4f(a.sigma, k0, n_pairs, g.cvec, 0.f, sg[r]);
+        if (a.chan_scale) {
+            load8f(a.chan_scale, e_out[r], g.d_in, g.cvec, 1.0f, cs[r]);
+        } else {
 #pragma unroll
-        for (int p = 0; p < 4; ++p) sg[r][p] = (k0 + p < n_pairs) ? a.sigma[k0 + p] : 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float v[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int j = e_out[r] + 2 * i + h;
-                v[h] = (j < g.d_in) ? __fdiv_rn(float(a.signs[j]) * a.inv_sqrt_b, a.chan_scale ? a.chan_scale[j] : 1.0f) : 0.f;
-            }
-            mcol[r][i] = pack2(v[0], v[1]);
+            for (int e = 0; e < 8; ++e) cs[r][e] = 1.0f;
         }
+        load8s(a.signs, e_out[r], g.d_in, g.cvec, sgn[r]);
     }
+    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
+    f32x2 mcol[4][4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            mcol[r][i] = pack2(__fdiv_rn(sgn[r][2 * i] * a.inv_sqrt_b, cs[r][2 * i]),
+                               __fdiv_rn(sgn[r][2 * i + 1] * a.inv_sqrt_b, cs[r][2 * i + 1]));
     __syncthreads();
 
     int buf = 0;
@@ -1082,7 +1156,15 @@ RowGeom make_geom(const qamw_params* p, const void* W) {
     const size_t esz = g.w_bf16 ? 2 : 4;
     g.vec = (p->d_in % 8 == 0) && (reinterpret_cast<uintptr_t>(W) % 16 == 0) && ((size_t(p->w_row_stride) * esz) % 16 == 0);
     g.w_row_stride = p->w_row_stride;
+    g.cvec = 0;
     return g;
+}
+
+// Per-column constant arrays allow vector loads: d_in a multiple of 8, floats 16-byte and signs
+// 8-byte aligned.
+int const_vec_ok(const qamw_params* p, const float* chan_scale, const int8_t* signs, const float* sigma) {
+    auto al = [](const void* q, uintptr_t a) { return reinterpret_cast<uintptr_t>(q) % a == 0; };
+    return (p->d_in % 8 == 0) && al(chan_scale, 16) && al(signs, 8) && al(sigma, 16);
 }
 
 int sm_count() {
@@ -1237,6 +1319,7 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     if (p->d_out == 0) return QAMW_OK;
     EncodeArgs a;
     a.g = make_geom(p, W);
+    a.g.cvec = const_vec_ok(p, chan_scale, signs, sigma);
     a.W = W;
     a.chan_scale = chan_scale;
     a.signs = signs;
@@ -1279,6 +1362,7 @@ extern "C" int qamw_rotate(const void* W, const qamw_params* p, const float* cha
     if (p->d_out == 0) return QAMW_OK;
     AuxArgs a{};
     a.g = make_geom(p, W);
+    a.g.cvec = const_vec_ok(p, chan_scale, signs, nullptr);
     a.W = W;
     a.chan_scale = chan_scale;
     a.signs = signs;
@@ -1325,6 +1409,7 @@ extern "C" int qamw_calibrate(const void* W, const qamw_params* p, const float* 
     if (reinterpret_cast<uintptr_t>(workspace) % 8) return QAMW_ERR_ALIGN;
     AuxArgs a{};
     a.g = make_geom(p, W);
+    a.g.cvec = const_vec_ok(p, chan_scale, signs, nullptr);
     const CalibPlan c = calib_plan(p, a.g);
     if (workspace_bytes < c.bytes) return QAMW_ERR_NOMEM;
     a.W = W;
@@ -1412,6 +1497,7 @@ extern "C" int qamw_decode(const uint8_t* packed, const float* row_norm, const f
     if (p->d_out == 0) return QAMW_OK;
     DecodeArgs a;
     a.g = make_geom(p, nullptr);
+    a.g.cvec = const_vec_ok(p, chan_scale, signs, sigma);
     a.g.vec = (p->d_in % 8 == 0) && (reinterpret_cast<uintptr_t>(w_hat_bf16_out) % 16 == 0);
     a.packed = packed;
     a.packed_row_stride = p->packed_row_stride;
