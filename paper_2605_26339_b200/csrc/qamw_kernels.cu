@@ -30,6 +30,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <type_traits>
 
 #include "qamw_internal.h"
 
@@ -408,7 +409,8 @@ __device__ __forceinline__ void col_factors(const ColRaw& c, f32x2 (&t)[4][4]) {
 // buffers).
 template <bool BF16, int LOG2B_T>
 __device__ __forceinline__ float front_half(const RawRow<BF16>& raw, const f32x2 (&t)[4][4], f32x2 (&P)[4][4],
-                                            const RowGeom& g, int group, int tid_g, double* red, int parity) {
+                                            const RowGeom& g, int group, int tid_g, double* red, int parity,
+                                            float& gn_out) {
     float x[4][8];
     raw_to_float<BF16>(raw, x);
     double ss = 0.0;
@@ -429,14 +431,20 @@ __device__ __forceinline__ float front_half(const RawRow<BF16>& raw, const f32x2
     double* slot = red + parity * 32;
     if ((tid_g & 31) == 0) slot[tid_g >> 5] = ss;
     group_barrier(group, g.tg);
-    double total = 0.0;
-    for (int w = 0; w < n_warps; ++w) total += slot[w];
-    return float(sqrt(total));
-}
-
-// g = f32(1 / (r * sqrt(b))), computed in double.
-__device__ __forceinline__ float inv_norm_factor(float r, int log2b) {
-    return float(1.0 / (double(r) * sqrt(double(1 << log2b))));
+    // one thread of the group turns the warp sums into r and g = f32(1 / (r sqrt(b))) (g = 0 for a
+    // zero or non-finite row); the others pick both up after a second barrier
+    float2* rg = reinterpret_cast<float2*>(slot + 16);
+    if (tid_g == 0) {
+        double total = 0.0;
+        for (int w = 0; w < n_warps; ++w) total += slot[w];
+        const float r = float(sqrt(total));
+        const float gn = (isfinite(r) && r > 0.f) ? float(1.0 / (double(r) * sqrt(double(1 << g.log2b)))) : 0.f;
+        *rg = make_float2(r, gn);
+    }
+    group_barrier(group, g.tg);
+    const float2 v = *rg;
+    gn_out = v.y;
+    return v.x;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -509,7 +517,7 @@ __device__ __noinline__ int search_exhaustive(const SearchSmem& s, float zx, flo
     return arg;
 }
 
-__device__ __noinline__ int search_overflow(const SearchSmem& s, uint2 rec, float zx, float zy) {
+__device__ __forceinline__ int search_overflow(const SearchSmem& s, uint2 rec, float zx, float zy) {
     const int off = int(rec.x >> 16), cnt = int(rec.y & 0xffffu);
     float best = INFINITY;
     int arg = 0;
@@ -517,25 +525,26 @@ __device__ __noinline__ int search_overflow(const SearchSmem& s, uint2 rec, floa
     return arg;
 }
 
-__device__ __forceinline__ int search_table(const SearchSmem& s, float zx, float zy) {
-    // beyond the table's reach (or NaN): exhaustive scan
-    if (!(fmaxf(fabsf(zx), fabsf(zy)) < 16000.0f)) return search_exhaustive(s, zx, zy);
-    const float fx = __fmaf_rn(zx, 256.0f, 2048.0f), fy = __fmaf_rn(zy, 256.0f, 2048.0f);
-    const int bx = min(max(int(fx), 0), 4095), by = min(max(int(fy), 0), 4095);
+// Table search for a point known to lie inside the table's reach (|z| < 16000, not NaN).
+__device__ __forceinline__ int search_cell(const SearchSmem& s, float zx, float zy) {
+    // fine bin = clamp(floor(z * 256 + 2048), 0, 4095); the conversion saturates negatives to 0
+    const unsigned bx = min(__float2uint_rz(__fmaf_rn(zx, 256.0f, 2048.0f)), 4095u);
+    const unsigned by = min(__float2uint_rz(__fmaf_rn(zy, 256.0f, 2048.0f)), 4095u);
     const int ix = s.lut[bx], iy = s.lut[by];
     const uint2 rec = s.cells[iy * s.grid + ix];
     const int k0 = int(rec.x & 0xffffu);
     if (k0 == 0xffff) return search_overflow(s, rec, zx, zy);
     const int k1 = int(rec.x >> 16), k2 = int(rec.y & 0xffffu), k3 = int(rec.y >> 16);
-    // The list is ascending and padded by repeating its last entry: a repeated slot needs no
-    // second read, its distance is the one just computed.
-    const float d0 = dist2(codeword(s, k0), zx, zy);
-    float d1 = d0;
-    if (k1 != k0) d1 = dist2(codeword(s, k1), zx, zy);
-    float d2 = d1;
-    if (k2 != k1) d2 = dist2(codeword(s, k2), zx, zy);
-    float d3 = d2;
-    if (k3 != k2) d3 = dist2(codeword(s, k3), zx, zy);
+    // The list is ascending and padded by repeating its last entry: a repeated slot is not read
+    // again (its distance equals the previous one and cannot win).
+    const float2 c0 = codeword(s, k0);
+    float2 c1 = c0, c2, c3;
+    if (k1 != k0) c1 = codeword(s, k1);
+    c2 = c1;
+    if (k2 != k1) c2 = codeword(s, k2);
+    c3 = c2;
+    if (k3 != k2) c3 = codeword(s, k3);
+    const float d0 = dist2(c0, zx, zy), d1 = dist2(c1, zx, zy), d2 = dist2(c2, zx, zy), d3 = dist2(c3, zx, zy);
     // lowest slot (= lowest index) among equal distances
     float best = d0;
     int arg = k0;
@@ -545,9 +554,16 @@ __device__ __forceinline__ int search_table(const SearchSmem& s, float zx, float
     return arg;
 }
 
-// Position of pair k in the index staging row: 16 halfwords of padding after every 64 pairs keep
-// the 8-byte stores of a warp (eight runs of 32 bytes, 128 bytes apart) on distinct banks.
-__device__ __forceinline__ int stage_pos(int k) { return k + ((k >> 6) << 4); }
+__device__ __noinline__ int search_table(const SearchSmem& s, float zx, float zy) {
+    // beyond the table's reach (or NaN): exhaustive scan
+    if (!(fmaxf(fabsf(zx), fabsf(zy)) < 16000.0f)) return search_exhaustive(s, zx, zy);
+    return search_cell(s, zx, zy);
+}
+
+// Index staging: the 4 indices of an octet are staged as one 64-bit value (index p at bits
+// [p*B, (p+1)*B)).  Octet o sits in 8-byte slot o + 4*(o/16): the 32 bytes of padding after every
+// 16 octets keep the stores of a warp (eight runs of 32 bytes, 128 bytes apart) on distinct banks.
+__device__ __forceinline__ int stage_slot(int o) { return o + ((o >> 4) << 2); }
 
 // ---------------------------------------------------------------------------------------------
 // encode kernel
@@ -640,62 +656,84 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
 
     const long long row_step = (long long)gridDim.x * g.groups;
     long long row = (long long)blockIdx.x * g.groups + group;
-    const unsigned div_magic = 0xffffffffu / unsigned(a.log2K) + 1u;  // ceil(2^32 / B)
-
-    RawRow<BF16> raw;
-    if (row < g.d_out) load_row<BF16, LOG2B_T>(raw, a.W, row, g, tid_g);
-    int parity = 0;
-    for (; row < g.d_out; row += row_step, parity ^= 1) {
-        RawRow<BF16> nxt;
-        const long long next_row = row + row_step;
-        if (next_row < g.d_out) load_row<BF16, LOG2B_T>(nxt, a.W, next_row, g, tid_g);
-
-        f32x2 P[4][4];
-        const float r = front_half<BF16, LOG2B_T>(raw, t, P, g, group, tid_g, red, parity);
-        const bool finite = isfinite(r);
-        if (tid_g == 0) {
-            a.row_norm[row] = r;
-            if (!finite && a.status) atomicOr(a.status, 1);
-        }
-        const bool live = finite && r > 0.f;  // zero or non-finite rows are encoded as the origin
-        const float gn = live ? inv_norm_factor(r, g.log2b) : 0.f;
-        const f32x2 gn2 = pack2(gn, gn);
-
+    const int B = a.log2K, B4 = 4 * a.log2K;
+    const unsigned div_magic = 0xffffffffu / unsigned(B4) + 1u;  // ceil(2^32 / (4B))
+    const int n_oct = (n_pairs + 3) >> 2;
+    unsigned long long* oct_s = reinterpret_cast<unsigned long long*>(idx_s);
+    // |z| <= q (1 + eps) because |y| <= 1 for a unit row: only a thread with a huge reciprocal pair
+    // scale can leave the table's reach and needs the checked search
+    bool risky = false;
 #pragma unroll
-        for (int rr = 0; rr < 4; ++rr) {
-            const int k0 = k0s[rr];
-            if (k0 < n_pairs) {
-                uint32_t id[4];
+    for (int r = 0; r < 4; ++r)
 #pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    float yx, yy;
-                    unpack2(mul2(P[rr][p], gn2), yx, yy);
-                    float zx = __fmul_rn(yx, q[rr][p]), zy = __fmul_rn(yy, q[rr][p]);
-                    if (!live) zx = zy = 0.f;
-                    id[p] = uint32_t(a.brute ? search_exhaustive(s, zx, zy) : search_table(s, zx, zy));
+        for (int p = 0; p < 4; ++p) risky |= !(q[r][p] < 15000.0f);
+
+    // The row loop exists in three variants chosen once per block, so that the common one carries
+    // no call to the rarely needed searches: 0 = table search, 1 = table search with the reach
+    // check, 2 = exhaustive search.
+    const int any_risky = __syncthreads_or(risky ? 1 : 0);
+    auto rows = [&](auto mode_tag) {
+        constexpr int MODE = decltype(mode_tag)::value;
+        int parity = 0;
+        for (; row < g.d_out; row += row_step, parity ^= 1) {
+            RawRow<BF16> raw;
+            load_row<BF16, LOG2B_T>(raw, a.W, row, g, tid_g);
+
+            f32x2 P[4][4];
+            float gn;
+            const float r = front_half<BF16, LOG2B_T>(raw, t, P, g, group, tid_g, red, parity, gn);
+            if (tid_g == 0) {
+                a.row_norm[row] = r;
+                if (!isfinite(r) && a.status) atomicOr(a.status, 1);
+            }
+            // zero or non-finite rows have g = 0: every pair becomes the origin (0 * inf is avoided
+            // because such rows are rotated like any other and only then multiplied by 0; a NaN
+            // product is mapped to the origin below)
+            const bool live = gn != 0.f;
+            const f32x2 gn2 = pack2(gn, gn);
+
+    #pragma unroll
+            for (int rr = 0; rr < 4; ++rr) {
+                const int k0 = k0s[rr];
+                if (k0 < n_pairs) {
+                    uint32_t id[4];
+    #pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        float yx, yy;
+                        unpack2(mul2(P[rr][p], gn2), yx, yy);
+                        float zx = __fmul_rn(yx, q[rr][p]), zy = __fmul_rn(yy, q[rr][p]);
+                        if (!live) zx = zy = 0.f;
+                        int v;
+                        if (MODE == 2) v = search_exhaustive(s, zx, zy);
+                        else if (MODE == 1) v = search_table(s, zx, zy);
+                        else v = search_cell(s, zx, zy);
+                        id[p] = (k0 + p < n_pairs) ? uint32_t(v) : 0u;
+                    }
+                    const uint32_t lo = id[0] | (id[1] << B), hi = id[2] | (id[3] << B);
+                    oct_s[stage_slot(k0 >> 2)] = (unsigned long long)lo | ((unsigned long long)hi << (2 * B));
                 }
-                *reinterpret_cast<uint2*>(idx_s + stage_pos(k0)) = make_uint2(id[0] | (id[1] << 16), id[2] | (id[3] << 16));
             }
-        }
-        group_barrier(group, g.tg);
+            group_barrier(group, g.tg);
 
-        // bit packing: index k occupies bits [k*B, (k+1)*B) of the row stream (LSB first)
-        uint32_t* out = reinterpret_cast<uint32_t*>(a.packed + row * a.packed_row_stride);
-        const int B = a.log2K;
-        for (int w = tid_g; w < a.row_words; w += g.tg) {
-            const unsigned bit0 = unsigned(w) * 32u;
-            int k = int(__umulhi(bit0, div_magic));  // floor(bit0 / B)
-            uint32_t word = 0;
-            for (; k < n_pairs; ++k) {
-                const int sh = k * B - int(bit0);
-                if (sh >= 32) break;
-                const uint32_t v = idx_s[stage_pos(k)];
-                word |= sh >= 0 ? (v << sh) : (v >> (-sh));
+            // bit packing: octet o occupies bits [o*4B, (o+1)*4B) of the row stream (LSB first)
+            uint32_t* out = reinterpret_cast<uint32_t*>(a.packed + row * a.packed_row_stride);
+            for (int w = tid_g; w < a.row_words; w += g.tg) {
+                const unsigned bit0 = unsigned(w) * 32u;
+                int o = int(__umulhi(bit0, div_magic));  // floor(bit0 / (4B))
+                uint32_t word = 0;
+                for (; o < n_oct; ++o) {
+                    const int sh = o * B4 - int(bit0);
+                    if (sh >= 32) break;
+                    const unsigned long long v = oct_s[stage_slot(o)];
+                    word |= sh >= 0 ? uint32_t(v << sh) : uint32_t(v >> (-sh));
+                }
+                out[w] = word;
             }
-            out[w] = word;
         }
-        raw = nxt;
-    }
+    };
+    if (a.brute) rows(std::integral_constant<int, 2>{});
+    else if (any_risky) rows(std::integral_constant<int, 1>{});
+    else rows(std::integral_constant<int, 0>{});
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -763,10 +801,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) aux_kernel(const AuxArgs a) {
             load_row<BF16, LOG2B_T>(nxt, a.W, row_next, g, tid_g);
         }
         f32x2 P[4][4];
-        const float r = front_half<BF16, LOG2B_T>(raw, t, P, g, group, tid_g, red, parity);
-        const bool finite = isfinite(r);
-        if (!finite && a.status && tid_g == 0) atomicOr(a.status, 1);
-        const float gn = (finite && r > 0.f) ? inv_norm_factor(r, g.log2b) : 0.f;
+        float gn;
+        const float r = front_half<BF16, LOG2B_T>(raw, t, P, g, group, tid_g, red, parity, gn);
+        if (!isfinite(r) && a.status && tid_g == 0) atomicOr(a.status, 1);
         const f32x2 gn2 = pack2(gn, gn);
         if (a.mode == 0) {
             if (tid_g == 0) a.row_norm[row] = r;
