@@ -482,18 +482,43 @@ __device__ __forceinline__ void fill_codebook_copies(float2* dst, const float2* 
 // nearest-codeword search
 // ---------------------------------------------------------------------------------------------
 
-struct SearchSmem {
-    const unsigned char* cb;  // codebook copies, already offset to this lane's copy
-    int cb_shift;             // log2 of the byte distance between consecutive entries (3 + log2c)
-    const uint2* cells;       // grid*grid records
-    const uint16_t* overflow;
-    const uint8_t* lut;       // 4096 bytes
+// Shared-memory reads of the read-only tables, by 32-bit shared address.  Written as plain
+// (non-volatile) asm: the tables never change after the prologue's barrier, so these loads may be
+// scheduled freely around the stores to the staging buffers.
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ float2 lds_f32x2(uint32_t addr) {
+    float2 v;
+    asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds_u32x2(uint32_t addr) {
+    uint2 v;
+    asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
+    uint32_t v;
+    asm("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
+    uint32_t v;
+    asm("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+struct SearchSmem {       // all fields are shared-memory byte addresses
+    uint32_t cb;          // codebook copies, already offset to this lane's copy
+    int cb_shift;         // log2 of the byte distance between consecutive entries (3 + log2c)
+    uint32_t cells;       // grid*grid records of 8 bytes
+    uint32_t overflow;    // u16 lists
+    uint32_t lut;         // 4096 bytes
     int grid;
     int K;
 };
 
 __device__ __forceinline__ float2 codeword(const SearchSmem& s, int k) {
-    return *reinterpret_cast<const float2*>(s.cb + (size_t(k) << s.cb_shift));
+    return lds_f32x2(s.cb + (uint32_t(k) << s.cb_shift));
 }
 
 // Squared distance in direct form, one rounding per operation: (zx-cx)^2 + (zy-cy)^2.
@@ -521,7 +546,7 @@ __device__ __forceinline__ int search_overflow(const SearchSmem& s, uint2 rec, f
     const int off = int(rec.x >> 16), cnt = int(rec.y & 0xffffu);
     float best = INFINITY;
     int arg = 0;
-    for (int i = 0; i < cnt; ++i) consider(s, int(s.overflow[off + i]), zx, zy, best, arg);
+    for (int i = 0; i < cnt; ++i) consider(s, int(lds_u16(s.overflow + 2u * uint32_t(off + i))), zx, zy, best, arg);
     return arg;
 }
 
@@ -530,20 +555,13 @@ __device__ __forceinline__ int search_cell(const SearchSmem& s, float zx, float 
     // fine bin = clamp(floor(z * 256 + 2048), 0, 4095); the conversion saturates negatives to 0
     const unsigned bx = min(__float2uint_rz(__fmaf_rn(zx, 256.0f, 2048.0f)), 4095u);
     const unsigned by = min(__float2uint_rz(__fmaf_rn(zy, 256.0f, 2048.0f)), 4095u);
-    const int ix = s.lut[bx], iy = s.lut[by];
-    const uint2 rec = s.cells[iy * s.grid + ix];
+    const uint32_t ix = lds_u8(s.lut + bx), iy = lds_u8(s.lut + by);
+    const uint2 rec = lds_u32x2(s.cells + 8u * (iy * uint32_t(s.grid) + ix));
     const int k0 = int(rec.x & 0xffffu);
     if (k0 == 0xffff) return search_overflow(s, rec, zx, zy);
     const int k1 = int(rec.x >> 16), k2 = int(rec.y & 0xffffu), k3 = int(rec.y >> 16);
-    // The list is ascending and padded by repeating its last entry: a repeated slot is not read
-    // again (its distance equals the previous one and cannot win).
-    const float2 c0 = codeword(s, k0);
-    float2 c1 = c0, c2, c3;
-    if (k1 != k0) c1 = codeword(s, k1);
-    c2 = c1;
-    if (k2 != k1) c2 = codeword(s, k2);
-    c3 = c2;
-    if (k3 != k2) c3 = codeword(s, k3);
+    // The list is ascending and padded by repeating its last entry (a repeated slot cannot win).
+    const float2 c0 = codeword(s, k0), c1 = codeword(s, k1), c2 = codeword(s, k2), c3 = codeword(s, k3);
     const float d0 = dist2(c0, zx, zy), d1 = dist2(c1, zx, zy), d2 = dist2(c2, zx, zy), d3 = dist2(c3, zx, zy);
     // lowest slot (= lowest index) among equal distances
     float best = d0;
@@ -643,11 +661,11 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     __syncthreads();
 
     SearchSmem s;
-    s.cb = smem + 8 * (threadIdx.x & ((1 << a.log2c) - 1));
+    s.cb = smem_addr(smem) + 8u * (threadIdx.x & ((1 << a.log2c) - 1));
     s.cb_shift = 3 + a.log2c;
-    s.cells = reinterpret_cast<const uint2*>(table);
-    s.overflow = reinterpret_cast<const uint16_t*>(table + a.off_overflow);
-    s.lut = table + a.off_lut;
+    s.cells = smem_addr(table);
+    s.overflow = smem_addr(table + a.off_overflow);
+    s.lut = smem_addr(table + a.off_lut);
     s.grid = a.grid;
     s.K = a.K;
 
@@ -941,7 +959,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
     const int B = a.log2K;
     const uint32_t mask = (1u << B) - 1u;
     const uint32_t cb_stride = 8u << a.log2c;
-    const unsigned char* cb = smem + 8 * (threadIdx.x & ((1 << a.log2c) - 1));
+    const uint32_t cb = smem_addr(smem) + 8u * (threadIdx.x & ((1 << a.log2c) - 1));
     unsigned char* stage = smem + ((size_t(a.K) * 8) << a.log2c) + size_t(threadIdx.x >> 5) * 2 * a.stage_bytes;
 
     // first row on its way before anything else
@@ -1017,7 +1035,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
                     // pairs past the end of a row whose length is not a multiple of 8 have scale 0
-                    const float2 c = *reinterpret_cast<const float2*>(cb + id[p] * cb_stride);
+                    const float2 c = lds_f32x2(cb + id[p] * cb_stride);
                     P[r][p] = pack2(c.x * sg[r][p], c.y * sg[r][p]);
                 }
             } else {
