@@ -26,7 +26,7 @@
  *       t_j = f32(s_j) * sign_j;  x_j = f32(f32(W_ij) * t_j);
  *       r_i = f32(sqrt(sum_j (double)x_j^2));
  *       h   = f32 butterfly of x per block, stages 1, 2, 4, ..., b/2, (a, b) -> (a+b, a-b);
- *       y_j = f32(h_j * g),  g = f32(1 / ((double)r_i * sqrt((double)b)));
+ *       y_j = f32(h_j * g),  g = f32(c_b / r_i) (one f32 division),  c_b = f32(1 / sqrt((double)b));
  *       z   = f32(y * q_k),  q_k = f32(1 / (double)sigma_k);
  *       idx = argmin_c fma(dy, dy, dx*dx) in f32 with dx = z_x - c_x, dy = z_y - c_y,
  *             lowest index among equal distances.

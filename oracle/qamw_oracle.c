@@ -273,7 +273,8 @@ void orc_fwht_f64(double *x, int b) {
  *   (ii)  ss  = sum_j (double)x_j * (double)x_j   (j ascending, double)
  *         r   = f32( sqrt(ss) )
  *   (iii) h   = butterfly_f32(x) per block of b   (orc_fwht_f32)
- *   (iv)  g   = f32( 1 / ((double)r * sqrt((double)b)) );  y_j = f32(h_j * g)
+ *   (iv)  c_b = f32( 1 / sqrt((double)b) );  g = f32( c_b / r )  (one f32 division)
+ *         y_j = f32(h_j * g)
  *         r == 0  ->  y = 0   (Section 3.1 step 1: "encoded as a zero row")
  * Returns ORC_ERR_NONFINITE when r is not finite (y is then unspecified).
  */
@@ -295,7 +296,8 @@ int orc_front_row(const void *W_row, int w_dtype, int d_in, int b, const float *
         return ORC_OK;
     }
     for (int blk = 0; blk < d_in / b; ++blk) orc_fwht_f32(y_out + blk * b, b);
-    volatile float g = (float)(1.0 / ((double)r * sqrt((double)b)));
+    volatile float cb = (float)(1.0 / sqrt((double)b));
+    volatile float g = cb / r;
     for (int j = 0; j < d_in; ++j) {
         volatile float y = y_out[j] * g;
         y_out[j] = y;

@@ -431,14 +431,14 @@ __device__ __forceinline__ float front_half(const RawRow<BF16>& raw, const f32x2
     double* slot = red + parity * 32;
     if ((tid_g & 31) == 0) slot[tid_g >> 5] = ss;
     group_barrier(group, g.tg);
-    // one thread of the group turns the warp sums into r and g = f32(1 / (r sqrt(b))) (g = 0 for a
+    // one thread of the group turns the warp sums into r and g = f32(c_b / r), c_b = f32(1/sqrt(b)) (g = 0 for a
     // zero or non-finite row); the others pick both up after a second barrier
     float2* rg = reinterpret_cast<float2*>(slot + 16);
     if (tid_g == 0) {
         double total = 0.0;
         for (int w = 0; w < n_warps; ++w) total += slot[w];
         const float r = float(sqrt(total));
-        const float gn = (isfinite(r) && r > 0.f) ? float(1.0 / (double(r) * sqrt(double(1 << g.log2b)))) : 0.f;
+        const float gn = (isfinite(r) && r > 0.f) ? __fdiv_rn(float(1.0 / sqrt(double(1 << g.log2b))), r) : 0.f;
         *rg = make_float2(r, gn);
     }
     group_barrier(group, g.tg);
@@ -600,21 +600,28 @@ struct EncodeArgs {
     int K, log2K, grid;
     int log2c;               // log2 of the number of codebook copies in shared memory
     int brute;
+    float inv_sqrt_b;        // c_b = f32(1 / sqrt(b))
     uint8_t* packed;
     long long packed_row_stride;  // bytes
     int row_words;           // 32-bit words per packed row (stride / 4)
-    float* row_norm;
-    int32_t* status;
-    int idx_stride;          // u16 entries of index staging per group
+    int payload_words;       // words that hold index bits: ceil(row payload bytes / 4)
+    const float* row_norm;   // written by row_norm_kernel just before
 };
 
+constexpr int kStageSlotsPerWarp = 128 + 4 * 8;  // 128 octets of a warp plus their padding
+
+// Encoder proper.  The row norms are already in global memory, so the warps of a row share
+// nothing: a warp owns 1024 consecutive elements (whole Hadamard blocks), rotates them with
+// shuffles, searches its 512 pairs, stages the indices in its own piece of shared memory and
+// writes its 64*B bytes of the packed row.  No block-wide barrier after the prologue.
 template <bool BF16, int LOG2B_T>
 __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
     const RowGeom& g = a.g;
-    // shared memory: [codebook copies][table][red: groups x 64 doubles][idx: groups x idx_stride u16]
+    // shared memory: [codebook copies][table][index staging: one piece per warp]
     const int group = threadIdx.x / g.tg;
     const int tid_g = threadIdx.x - group * g.tg;
+    const int lane = threadIdx.x & 31;
     const int n_pairs = g.d_in >> 1;
     // all global loads of the prologue are issued before anything waits for one of them
     ColRaw craw;
@@ -647,18 +654,24 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
         }
     }
     const int table_pad = (a.table_bytes + 15) & ~15;
-    double* red_all = reinterpret_cast<double*>(table + table_pad);
-    uint16_t* idx_all = reinterpret_cast<uint16_t*>(table + table_pad + g.groups * 64 * sizeof(double));
+    unsigned long long* oct_s =
+        reinterpret_cast<unsigned long long*>(table + table_pad) + size_t(threadIdx.x >> 5) * kStageSlotsPerWarp;
 
     f32x2 t[4][4];
     col_factors(craw, t);
     // q_k = f32(1 / (double)sigma_k): the correctly rounded f32 reciprocal is the same number (the
     // exact quotient of two f32 is never within 2^-53 of an f32 rounding boundary unless it is exact)
+    bool risky = false;
 #pragma unroll
     for (int r = 0; r < 4; ++r)
 #pragma unroll
-        for (int p = 0; p < 4; ++p) q[r][p] = (k0s[r] + p < n_pairs) ? __frcp_rn(q[r][p]) : 0.f;
-    __syncthreads();
+        for (int p = 0; p < 4; ++p) {
+            q[r][p] = (k0s[r] + p < n_pairs) ? __frcp_rn(q[r][p]) : 0.f;
+            // |z| <= q (1 + eps) because |y| <= 1 for a unit row: only a huge reciprocal pair scale
+            // can carry a point beyond the table's reach
+            risky |= !(q[r][p] < 15000.0f);
+        }
+    const int any_risky = __syncthreads_or(risky ? 1 : 0);  // also the prologue's barrier
 
     SearchSmem s;
     s.cb = smem_addr(smem) + 8u * (threadIdx.x & ((1 << a.log2c) - 1));
@@ -669,53 +682,47 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     s.grid = a.grid;
     s.K = a.K;
 
-    double* red = red_all + group * 64;
-    uint16_t* idx_s = idx_all + size_t(group) * a.idx_stride;
-
     const long long row_step = (long long)gridDim.x * g.groups;
-    long long row = (long long)blockIdx.x * g.groups + group;
     const int B = a.log2K, B4 = 4 * a.log2K;
     const unsigned div_magic = 0xffffffffu / unsigned(B4) + 1u;  // ceil(2^32 / (4B))
     const int n_oct = (n_pairs + 3) >> 2;
-    unsigned long long* oct_s = reinterpret_cast<unsigned long long*>(idx_s);
-    // |z| <= q (1 + eps) because |y| <= 1 for a unit row: only a thread with a huge reciprocal pair
-    // scale can leave the table's reach and needs the checked search
-    bool risky = false;
+    const int warp_g = tid_g >> 5;                 // segment of the row this warp owns
+    const int oct0 = 128 * warp_g;                 // its first octet
+    const int seg_word0 = 16 * B * warp_g;         // its first packed word (64*B bytes per segment)
+    const bool last_seg = (warp_g + 1) * 1024 >= g.d_in;
+    int k_loc[4];                                   // staging slot of each held octet
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
-#pragma unroll
-        for (int p = 0; p < 4; ++p) risky |= !(q[r][p] < 15000.0f);
+    for (int r = 0; r < 4; ++r) k_loc[r] = stage_slot((k0s[r] >> 2) - oct0);
 
     // The row loop exists in three variants chosen once per block, so that the common one carries
     // no call to the rarely needed searches: 0 = table search, 1 = table search with the reach
     // check, 2 = exhaustive search.
-    const int any_risky = __syncthreads_or(risky ? 1 : 0);
     auto rows = [&](auto mode_tag) {
         constexpr int MODE = decltype(mode_tag)::value;
-        int parity = 0;
-        for (; row < g.d_out; row += row_step, parity ^= 1) {
+        for (long long row = (long long)blockIdx.x * g.groups + group; row < g.d_out; row += row_step) {
             RawRow<BF16> raw;
             load_row<BF16, LOG2B_T>(raw, a.W, row, g, tid_g);
-
-            f32x2 P[4][4];
-            float gn;
-            const float r = front_half<BF16, LOG2B_T>(raw, t, P, g, group, tid_g, red, parity, gn);
-            if (tid_g == 0) {
-                a.row_norm[row] = r;
-                if (!isfinite(r) && a.status) atomicOr(a.status, 1);
-            }
-            // zero or non-finite rows have g = 0: every pair becomes the origin (0 * inf is avoided
-            // because such rows are rotated like any other and only then multiplied by 0; a NaN
-            // product is mapped to the origin below)
-            const bool live = gn != 0.f;
+            const float r = __ldg(a.row_norm + row);
+            // g = f32(c_b / r); 0 for a zero or non-finite row, whose pairs all become the origin
+            const bool live = isfinite(r) && r > 0.f;
+            const float gn = live ? __fdiv_rn(a.inv_sqrt_b, r) : 0.f;
             const f32x2 gn2 = pack2(gn, gn);
-
-    #pragma unroll
+            f32x2 P[4][4];
+            {
+                float x[4][8];
+                raw_to_float<BF16>(raw, x);
+#pragma unroll
+                for (int rr = 0; rr < 4; ++rr)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) P[rr][i] = mul2(pack2(x[rr][2 * i], x[rr][2 * i + 1]), t[rr][i]);
+            }
+            fwht_regs<LOG2B_T>(P, g.log2b, tid_g);
+#pragma unroll
             for (int rr = 0; rr < 4; ++rr) {
                 const int k0 = k0s[rr];
                 if (k0 < n_pairs) {
                     uint32_t id[4];
-    #pragma unroll
+#pragma unroll
                     for (int p = 0; p < 4; ++p) {
                         float yx, yy;
                         unpack2(mul2(P[rr][p], gn2), yx, yy);
@@ -728,30 +735,100 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                         id[p] = (k0 + p < n_pairs) ? uint32_t(v) : 0u;
                     }
                     const uint32_t lo = id[0] | (id[1] << B), hi = id[2] | (id[3] << B);
-                    oct_s[stage_slot(k0 >> 2)] = (unsigned long long)lo | ((unsigned long long)hi << (2 * B));
+                    oct_s[k_loc[rr]] = (unsigned long long)lo | ((unsigned long long)hi << (2 * B));
                 }
             }
-            group_barrier(group, g.tg);
-
-            // bit packing: octet o occupies bits [o*4B, (o+1)*4B) of the row stream (LSB first)
+            __syncwarp();
+            // bit packing of the warp's segment: octet o occupies bits [o*4B, (o+1)*4B) (LSB first)
             uint32_t* out = reinterpret_cast<uint32_t*>(a.packed + row * a.packed_row_stride);
-            for (int w = tid_g; w < a.row_words; w += g.tg) {
-                const unsigned bit0 = unsigned(w) * 32u;
-                int o = int(__umulhi(bit0, div_magic));  // floor(bit0 / (4B))
+            for (int j = lane; j < 16 * B; j += 32) {
+                const int gw = seg_word0 + j;
+                if (gw >= a.payload_words) break;
+                const unsigned bit0 = unsigned(j) * 32u;
+                int o = int(__umulhi(bit0, div_magic));  // floor(bit0 / (4B)), local octet
                 uint32_t word = 0;
-                for (; o < n_oct; ++o) {
+                for (; oct0 + o < n_oct; ++o) {
                     const int sh = o * B4 - int(bit0);
                     if (sh >= 32) break;
                     const unsigned long long v = oct_s[stage_slot(o)];
                     word |= sh >= 0 ? uint32_t(v << sh) : uint32_t(v >> (-sh));
                 }
-                out[w] = word;
+                out[gw] = word;
             }
+            if (last_seg)  // padding up to the row stride is written as zero
+                for (int gw = a.payload_words + lane; gw < a.row_words; gw += 32) out[gw] = 0u;
+            __syncwarp();  // the staging piece is free again
         }
     };
     if (a.brute) rows(std::integral_constant<int, 2>{});
     else if (any_risky) rows(std::integral_constant<int, 1>{});
     else rows(std::integral_constant<int, 0>{});
+}
+
+// ---------------------------------------------------------------------------------------------
+// row-norm kernel: r_i = f32(sqrt(sum_j (double)x_ij^2)), x_ij = f32(W_ij * t_j)
+// ---------------------------------------------------------------------------------------------
+// Same thread geometry as the other row kernels (a thread owns 32 columns, its factors t stay in
+// registers, the next row is prefetched into registers).  The warps of a row meet at one barrier
+// per row; nobody waits for the result, which goes to global memory for the encoder proper.
+
+struct NormArgs {
+    RowGeom g;
+    const void* W;
+    const float* chan_scale;
+    const int8_t* signs;
+    float* row_norm;
+    int32_t* status;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(kMaxThreads, 1) row_norm_kernel(const NormArgs a) {
+    __shared__ double red_all[kMaxGroups * 64];
+    const RowGeom& g = a.g;
+    const int group = threadIdx.x / g.tg;
+    const int tid_g = threadIdx.x - group * g.tg;
+    double* red = red_all + group * 64;
+    f32x2 t[4][4];
+    {
+        ColRaw craw;
+        load_col_raw<0>(craw, a.chan_scale, a.signs, g.d_in, g.cvec, tid_g);
+        col_factors(craw, t);
+    }
+    const long long row_step = (long long)gridDim.x * g.groups;
+    long long row = (long long)blockIdx.x * g.groups + group;
+    RawRow<BF16> raw;
+    if (row < g.d_out) load_row<BF16, 0>(raw, a.W, row, g, tid_g);
+    const int n_warps = g.tg >> 5;
+    int parity = 0;
+    for (; row < g.d_out; row += row_step, parity ^= 1) {
+        RawRow<BF16> nxt;
+        if (row + row_step < g.d_out) load_row<BF16, 0>(nxt, a.W, row + row_step, g, tid_g);
+        float x[4][8];
+        raw_to_float<BF16>(raw, x);
+        double ss = 0.0;
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float p, c;
+                unpack2(mul2(pack2(x[r][2 * i], x[r][2 * i + 1]), t[r][i]), p, c);
+                const double pd = double(p), cd = double(c);
+                ss = fma(pd, pd, ss);
+                ss = fma(cd, cd, ss);
+            }
+        ss = warp_sum(ss);
+        double* slot = red + parity * 32;
+        if ((tid_g & 31) == 0) slot[tid_g >> 5] = ss;
+        group_barrier(group, g.tg);
+        if (tid_g == 0) {
+            double total = 0.0;
+            for (int w = 0; w < n_warps; ++w) total += slot[w];
+            const float r = float(sqrt(total));
+            a.row_norm[row] = r;
+            if (!isfinite(r) && a.status) atomicOr(a.status, 1);
+        }
+        raw = nxt;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1270,6 +1347,12 @@ int launch_encode(const EncodeArgs& a, int blocks, size_t smem, cudaStream_t st)
     return finish_launch("encode_kernel");
 }
 
+template <bool BF16>
+int launch_norm(const NormArgs& a, int blocks, cudaStream_t st) {
+    row_norm_kernel<BF16><<<blocks, a.g.tg * a.g.groups, 0, st>>>(a);
+    return finish_launch("row_norm_kernel");
+}
+
 template <bool BF16, int LOG2B_T>
 int launch_aux(const AuxArgs& a, int blocks, cudaStream_t st) {
     aux_kernel<BF16, LOG2B_T><<<blocks, a.g.tg * a.g.groups, 0, st>>>(a);
@@ -1391,17 +1474,27 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     a.packed = packed_out;
     a.packed_row_stride = p->packed_row_stride;
     a.row_words = int(p->packed_row_stride / 4);
+    a.payload_words = int((row_bytes + 3) / 4);
     a.row_norm = row_norm_out;
-    a.status = status_out;
-    const int n_pairs = p->d_in / 2;
-    a.idx_stride = ((n_pairs + (n_pairs >> 6) * 16 + 7) / 8) * 8 + 24;
-    const size_t fixed = ((size_t(a.table_bytes) + 15) & ~size_t(15)) + size_t(a.g.groups) * 64 * sizeof(double) +
-                         size_t(a.g.groups) * a.idx_stride * 2;
+    a.inv_sqrt_b = float(1.0 / std::sqrt(double(p->block)));
+    const size_t fixed = ((size_t(a.table_bytes) + 15) & ~size_t(15)) +
+                         size_t(a.g.groups) * (a.g.tg / 32) * kStageSlotsPerWarp * 8;
     if (fixed + size_t(p->K) * 8 > kSmemLimit) return QAMW_ERR_NOMEM;
     a.log2c = pick_log2_copies(p->K, kSmemLimit - fixed);
     const size_t smem = fixed + (size_t(p->K) * 8 << a.log2c);
     const int blocks = std::max(1, std::min(sm_count(), (p->d_out + a.g.groups - 1) / a.g.groups));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    {   // row norms first: the encoder proper reads them from row_norm_out
+        NormArgs n;
+        n.g = a.g;
+        n.W = W;
+        n.chan_scale = chan_scale;
+        n.signs = signs;
+        n.row_norm = row_norm_out;
+        n.status = status_out;
+        rc = a.g.w_bf16 ? launch_norm<true>(n, blocks, st) : launch_norm<false>(n, blocks, st);
+        if (rc) return rc;
+    }
 #define CALL(LB)                                                                  \
     rc = a.g.w_bf16 ? launch_encode<true, LB>(a, blocks, smem, st) : launch_encode<false, LB>(a, blocks, smem, st)
     QAMW_DISPATCH_LOG2B(a.g.log2b, CALL)
