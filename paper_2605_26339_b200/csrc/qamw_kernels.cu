@@ -703,9 +703,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
             RawRow<BF16> raw;
             load_row<BF16, LOG2B_T>(raw, a.W, row, g, tid_g);
             const float r = __ldg(a.row_norm + row);
-            // g = f32(c_b / r); 0 for a zero or non-finite row, whose pairs all become the origin
-            const bool live = isfinite(r) && r > 0.f;
-            const float gn = live ? __fdiv_rn(a.inv_sqrt_b, r) : 0.f;
+            // g = f32(c_b / r); 0 for a zero row (all its pairs become the origin, 0 * 0) and for a
+            // non-finite row (its indices are unspecified; the searches accept any input)
+            const float gn = (isfinite(r) && r > 0.f) ? __fdiv_rn(a.inv_sqrt_b, r) : 0.f;
             const f32x2 gn2 = pack2(gn, gn);
             f32x2 P[4][4];
             {
@@ -726,8 +726,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                     for (int p = 0; p < 4; ++p) {
                         float yx, yy;
                         unpack2(mul2(P[rr][p], gn2), yx, yy);
-                        float zx = __fmul_rn(yx, q[rr][p]), zy = __fmul_rn(yy, q[rr][p]);
-                        if (!live) zx = zy = 0.f;
+                        const float zx = __fmul_rn(yx, q[rr][p]), zy = __fmul_rn(yy, q[rr][p]);
                         int v;
                         if (MODE == 2) v = search_exhaustive(s, zx, zy);
                         else if (MODE == 1) v = search_table(s, zx, zy);
@@ -746,12 +745,23 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                 if (gw >= a.payload_words) break;
                 const unsigned bit0 = unsigned(j) * 32u;
                 int o = int(__umulhi(bit0, div_magic));  // floor(bit0 / (4B)), local octet
-                uint32_t word = 0;
-                for (; oct0 + o < n_oct; ++o) {
-                    const int sh = o * B4 - int(bit0);
-                    if (sh >= 32) break;
-                    const unsigned long long v = oct_s[stage_slot(o)];
-                    word |= sh >= 0 ? uint32_t(v << sh) : uint32_t(v >> (-sh));
+                uint32_t word;
+                if (B4 >= 32) {
+                    // an octet is at least as wide as a word: the word takes bits from octet o and,
+                    // if it reaches past it, from octet o + 1 (slots past the row read as garbage
+                    // only into bits that the caller's row payload does not contain)
+                    const int sh = int(bit0) - o * B4;  // 0 <= sh < 4B
+                    const unsigned long long v0 = oct_s[stage_slot(o)];
+                    const unsigned long long v1 = (oct0 + o + 1 < n_oct) ? oct_s[stage_slot(o + 1)] : 0ull;
+                    word = uint32_t(v0 >> sh) | uint32_t((v1 << (B4 - sh)) & 0xffffffffull);
+                } else {
+                    word = 0;
+                    for (; oct0 + o < n_oct; ++o) {
+                        const int sh = o * B4 - int(bit0);
+                        if (sh >= 32) break;
+                        const unsigned long long v = oct_s[stage_slot(o)];
+                        word |= sh >= 0 ? uint32_t(v << sh) : uint32_t(v >> (-sh));
+                    }
                 }
                 out[gw] = word;
             }
