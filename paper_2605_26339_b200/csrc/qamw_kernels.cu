@@ -546,6 +546,7 @@ __device__ __forceinline__ int search_overflow(const SearchSmem& s, uint2 rec, f
     const int off = int(rec.x >> 16), cnt = int(rec.y & 0xffffu);
     float best = INFINITY;
     int arg = 0;
+#pragma unroll 1
     for (int i = 0; i < cnt; ++i) consider(s, int(lds_u16(s.overflow + 2u * uint32_t(off + i))), zx, zy, best, arg);
     return arg;
 }
@@ -657,6 +658,11 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     unsigned long long* oct_s =
         reinterpret_cast<unsigned long long*>(table + table_pad) + size_t(threadIdx.x >> 5) * kStageSlotsPerWarp;
 
+    // lane-private staging of the thread's sixteen points: [slot * 4 + p][lane] float2, after the index staging
+    float2* zst = reinterpret_cast<float2*>(reinterpret_cast<unsigned long long*>(table + table_pad) +
+                                            size_t(blockDim.x >> 5) * kStageSlotsPerWarp) +
+                  size_t(threadIdx.x >> 5) * 512 + lane;
+
     f32x2 t[4][4];
     col_factors(craw, t);
     // q_k = f32(1 / (double)sigma_k): the correctly rounded f32 reciprocal is the same number (the
@@ -690,9 +696,6 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     const int oct0 = 128 * warp_g;                 // its first octet
     const int seg_word0 = 16 * B * warp_g;         // its first packed word (64*B bytes per segment)
     const bool last_seg = (warp_g + 1) * 1024 >= g.d_in;
-    int k_loc[4];                                   // staging slot of each held octet
-#pragma unroll
-    for (int r = 0; r < 4; ++r) k_loc[r] = stage_slot((k0s[r] >> 2) - oct0);
 
     // The row loop exists in three variants chosen once per block, so that the common one carries
     // no call to the rarely needed searches: 0 = table search, 1 = table search with the reach
@@ -717,25 +720,33 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                     for (int i = 0; i < 4; ++i) P[rr][i] = mul2(pack2(x[rr][2 * i], x[rr][2 * i + 1]), t[rr][i]);
             }
             fwht_regs<LOG2B_T>(P, g.log2b, tid_g);
+            // The sixteen points of the thread go through a lane-private piece of shared memory, so
+            // that the search exists once in the instruction stream: a fully unrolled row loop does
+            // not fit the instruction cache, and fetch stalls then cost more than the extra
+            // shared-memory round trip.
 #pragma unroll
-            for (int rr = 0; rr < 4; ++rr) {
-                const int k0 = k0s[rr];
-                if (k0 < n_pairs) {
-                    uint32_t id[4];
+            for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
-                    for (int p = 0; p < 4; ++p) {
-                        float yx, yy;
-                        unpack2(mul2(P[rr][p], gn2), yx, yy);
-                        const float zx = __fmul_rn(yx, q[rr][p]), zy = __fmul_rn(yy, q[rr][p]);
-                        int v;
-                        if (MODE == 2) v = search_exhaustive(s, zx, zy);
-                        else if (MODE == 1) v = search_table(s, zx, zy);
-                        else v = search_cell(s, zx, zy);
-                        id[p] = (k0 + p < n_pairs) ? uint32_t(v) : 0u;
-                    }
-                    const uint32_t lo = id[0] | (id[1] << B), hi = id[2] | (id[3] << B);
-                    oct_s[k_loc[rr]] = (unsigned long long)lo | ((unsigned long long)hi << (2 * B));
+                for (int p = 0; p < 4; ++p) {
+                    float yx, yy;
+                    unpack2(mul2(P[rr][p], gn2), yx, yy);
+                    zst[(rr * 4 + p) * 32] = make_float2(__fmul_rn(yx, q[rr][p]), __fmul_rn(yy, q[rr][p]));
                 }
+#pragma unroll 1
+            for (int rr = 0; rr < 4; ++rr) {
+                const int k0 = 4 * Layout<LOG2B_T>::octet_after(tid_g, rr);
+                if (k0 >= n_pairs) continue;
+                unsigned long long packed4 = 0ull;
+#pragma unroll 1
+                for (int p = 0; p < 4; ++p) {
+                    const float2 z = zst[(rr * 4 + p) * 32];
+                    int v;
+                    if (MODE == 2) v = search_exhaustive(s, z.x, z.y);
+                    else if (MODE == 1) v = search_table(s, z.x, z.y);
+                    else v = search_cell(s, z.x, z.y);
+                    if (k0 + p < n_pairs) packed4 |= (unsigned long long)uint32_t(v) << (p * B);
+                }
+                oct_s[stage_slot((k0 >> 2) - oct0)] = packed4;
             }
             __syncwarp();
             // bit packing of the warp's segment: octet o occupies bits [o*4B, (o+1)*4B) (LSB first)
@@ -1402,10 +1413,11 @@ extern "C" int qamw_codebook_create(const float* codebook_host, int K, int grid,
     if (grid < 0 || grid > 255) return QAMW_ERR_ARG;
     *out = nullptr;
     SearchTable t;
-    // The encoder's shared memory also holds several codebook copies (at least 64 KB worth, two
-    // copies for K = 4096) and about 24 KB of per-group scratch: the table gets what is left of
-    // the 227 KB of one SM.
-    const size_t budget = size_t(227 - 24) * 1024 - std::max(size_t(64) * 1024, size_t(K) * 16);
+    // The encoder's shared memory also holds 84 KB of per-warp staging (16 warps x (1.25 KB of
+    // indices + 4 KB of points)) and the codebook in four bank-separated copies (one copy for
+    // K = 4096): the table gets what is left of the 227 KB of one SM.
+    const size_t copies = K <= 2048 ? 4 : 1;
+    const size_t budget = kSmemLimit - size_t(16) * (kStageSlotsPerWarp * 8 + 512 * 8) - size_t(K) * 8 * copies;
     if (!choose_search_table(codebook_host, K, grid, budget, &t)) return QAMW_ERR_NOMEM;
     qamw_codebook* cb = new (std::nothrow) qamw_codebook();
     if (!cb) return QAMW_ERR_NOMEM;
@@ -1488,7 +1500,7 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     a.row_norm = row_norm_out;
     a.inv_sqrt_b = float(1.0 / std::sqrt(double(p->block)));
     const size_t fixed = ((size_t(a.table_bytes) + 15) & ~size_t(15)) +
-                         size_t(a.g.groups) * (a.g.tg / 32) * kStageSlotsPerWarp * 8;
+                         size_t(a.g.groups) * (a.g.tg / 32) * (kStageSlotsPerWarp * 8 + 512 * 8);
     if (fixed + size_t(p->K) * 8 > kSmemLimit) return QAMW_ERR_NOMEM;
     a.log2c = pick_log2_copies(p->K, kSmemLimit - fixed);
     const size_t smem = fixed + (size_t(p->K) * 8 << a.log2c);
