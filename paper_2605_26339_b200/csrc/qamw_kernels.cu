@@ -965,26 +965,27 @@ __global__ void __launch_bounds__(kMaxThreads, 1) aux_kernel(const AuxArgs a) {
     }
 }
 
-// sigma_k from the per-group partial sums.  A block owns 32 pair positions; its 8 warps each add
-// a contiguous slice of the groups in ascending order and the 8 slice sums are then added in
-// ascending order, so the result does not depend on timing.
-__global__ void __launch_bounds__(256) calibrate_finish_kernel(const double* partial, int total_groups, int pair_stride,
-                                                               int n_pairs, int d_in, float* sigma_out) {
-    __shared__ double part_sum[8][32], part_used[8];
+// sigma_k from the per-group partial sums.  A block owns 32 pair positions; its 32 warps each add
+// a contiguous slice of the groups in ascending order (eight loads in flight at a time) and the 32
+// slice sums are then added in ascending order, so the result does not depend on timing.
+constexpr int kFinishSlices = 32;
+__global__ void __launch_bounds__(32 * kFinishSlices) calibrate_finish_kernel(const double* partial, int total_groups,
+                                                                            int pair_stride, int n_pairs, int d_in,
+                                                                            float* sigma_out) {
+    __shared__ double part_sum[kFinishSlices][32], part_used[kFinishSlices];
     const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
     const int k = blockIdx.x * 32 + lane;
-    const int per = (total_groups + 7) / 8;
+    const int per = (total_groups + kFinishSlices - 1) / kFinishSlices;
     const int g0 = min(total_groups, slice * per), g1 = min(total_groups, g0 + per);
     double sum = 0.0;
     if (k < n_pairs) {
         int gidx = g0;
-        for (; gidx + 4 <= g1; gidx += 4) {
-            const double v0 = partial[size_t(gidx) * pair_stride + k], v1 = partial[size_t(gidx + 1) * pair_stride + k];
-            const double v2 = partial[size_t(gidx + 2) * pair_stride + k], v3 = partial[size_t(gidx + 3) * pair_stride + k];
-            sum += v0;
-            sum += v1;
-            sum += v2;
-            sum += v3;
+        for (; gidx + 8 <= g1; gidx += 8) {
+            double v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = partial[size_t(gidx + u) * pair_stride + k];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) sum += v[u];
         }
         for (; gidx < g1; ++gidx) sum += partial[size_t(gidx) * pair_stride + k];
     }
@@ -997,7 +998,7 @@ __global__ void __launch_bounds__(256) calibrate_finish_kernel(const double* par
     __syncthreads();
     if (slice == 0 && k < n_pairs) {
         double s = 0.0, u = 0.0;
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < kFinishSlices; ++i) {
             s += part_sum[i][lane];
             u += part_used[i];
         }
@@ -1217,7 +1218,7 @@ __device__ __forceinline__ void dist_load(const void* W, long long w_row_stride,
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(kDistThreads) distortion_kernel(const void* W, long long w_row_stride,
+__global__ void __launch_bounds__(kDistThreads, 6) distortion_kernel(const void* W, long long w_row_stride,
                                                                   const __nv_bfloat16* What, const float* act_rms,
                                                                   int d_out, int d_in, int vec, double* out4) {
     const int col_tiles = (d_in + 8 * kDistThreads - 1) / (8 * kDistThreads);
@@ -1233,12 +1234,12 @@ __global__ void __launch_bounds__(kDistThreads) distortion_kernel(const void* W,
 #pragma unroll
         for (int e = 0; e < 8; ++e) E[e] = Q[e] = 0.0;
         int row = r0;
-        for (; row + 4 <= r1; row += 4) {  // four rows in flight
-            float w[4][8], h[4][8];
+        for (; row + 2 <= r1; row += 2) {  // two rows in flight per thread, eight blocks per SM
+            float w[2][8], h[2][8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) dist_load<BF16>(W, w_row_stride, What, row + u, j0, d_in, vec, w[u], h[u]);
+            for (int u = 0; u < 2; ++u) dist_load<BF16>(W, w_row_stride, What, row + u, j0, d_in, vec, w[u], h[u]);
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < 2; ++u)
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const double wd = double(w[u][e]), d = wd - double(h[u][e]);
@@ -1596,7 +1597,7 @@ extern "C" int qamw_calibrate(const void* W, const qamw_params* p, const float* 
 #undef CALL
     if (rc) return rc;
     const int n_pairs = p->d_in / 2;
-    calibrate_finish_kernel<<<(n_pairs + 31) / 32, 256, 0, st>>>(a.partial, c.total_groups, c.pair_stride, n_pairs,
+    calibrate_finish_kernel<<<(n_pairs + 31) / 32, 32 * kFinishSlices, 0, st>>>(a.partial, c.total_groups, c.pair_stride, n_pairs,
                                                                   p->d_in, sigma_out);
     return finish_launch("calibrate_finish_kernel");
 }
@@ -1714,7 +1715,7 @@ extern "C" int qamw_distortion(const void* W, const void* w_hat_bf16, const floa
                     ((size_t(p->w_row_stride) * esz) % 16 == 0) && (reinterpret_cast<uintptr_t>(w_hat_bf16) % 16 == 0);
     const long long items = (long long)((p->d_in + 8 * kDistThreads - 1) / (8 * kDistThreads)) *
                             ((p->d_out + kDistRows - 1) / kDistRows);
-    const int blocks = int(std::max<long long>(1, std::min<long long>(16LL * sm_count(), items)));
+    const int blocks = int(std::max<long long>(1, std::min<long long>(32LL * sm_count(), items)));
     if (p->w_dtype == QAMW_DTYPE_BF16)
         distortion_kernel<true><<<blocks, kDistThreads, 0, st>>>(W, p->w_row_stride,
                                                                  static_cast<const __nv_bfloat16*>(w_hat_bf16), act_rms,
