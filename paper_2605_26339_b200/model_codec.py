@@ -14,6 +14,29 @@ from . import binding as q
 from . import synth
 
 
+def shard_layers(n_layers: int, rank: int, world: int) -> List[int]:
+    """Layers owned by `rank` when a model is split over `world` devices: whole layers, round robin.
+    Every matrix is independent given its own scales and sigma, so no data crosses devices."""
+    if not (0 <= rank < world):
+        raise ValueError("rank must be in [0, world)")
+    return list(range(rank, n_layers, world))
+
+
+def combine_distortion(sums4: torch.Tensor, n_weights: int, group=None) -> Dict[str, float]:
+    """Model-wide error figures from per-rank sums [sum e^2, sum w^2, sum r^2 e^2, sum r^2 w^2]:
+    the only cross-device step of the codec, one all-reduce of five numbers (skipped when
+    torch.distributed is not initialised)."""
+    import torch.distributed as dist
+
+    v = torch.cat([sums4.detach().to(torch.float64).reshape(4), torch.tensor([float(n_weights)], dtype=torch.float64,
+                                                                             device=sums4.device)])
+    if dist.is_available() and dist.is_initialized():
+        dist.all_reduce(v, op=dist.ReduceOp.SUM, group=group)
+    d = v.cpu().numpy()
+    return {"rho_w": float(np.sqrt(d[0] / d[1])), "rho_o_diag": float(np.sqrt(d[2] / d[3])),
+            "mse": float(d[0] / d[4]), "n_weights": int(d[4])}
+
+
 @dataclass
 class MatrixSlot:
     """Device-resident state of one weight matrix."""
@@ -120,7 +143,6 @@ class ModelCodec:
         # calibrate = 2 kernels, encode 1, decode 1, distortion 1 (its memset is not a kernel of ours)
         return 5 * len(self.slots)
 
-    def totals(self) -> Dict[str, float]:
-        d = torch.stack([s.dist for s in self.slots]).sum(0).cpu().numpy()
-        return {"rho_w": float(np.sqrt(d[0] / d[1])), "rho_o_diag": float(np.sqrt(d[2] / d[3])),
-                "mse": float(d[0] / self.n_weights)}
+    def totals(self, group=None) -> Dict[str, float]:
+        """Error figures over all matrices of all ranks (see combine_distortion)."""
+        return combine_distortion(torch.stack([s.dist for s in self.slots]).sum(0), self.n_weights, group)

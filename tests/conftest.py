@@ -12,6 +12,12 @@ GOLDEN = os.path.join(ROOT, "tests", "golden")
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200 with -m gpu)")
+    # the shared library is built in-tree (nvcc cross-compiles without a GPU); a box without nvcc
+    # uses the copy that travelled with the repository
+    import shutil
+    from paper_2605_26339_b200 import build as lib_build
+    if lib_build.needs_build() and (shutil.which("nvcc") or os.path.exists("/usr/local/cuda/bin/nvcc")):
+        lib_build.build()
 
 
 def load_golden_codebook(K: int) -> np.ndarray:
