@@ -298,7 +298,7 @@ def run_ours(args):
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": workload_label(spec), "weights_per_gpu": n_w, "matrices": len(mc.slots),
+        "config": {"workload": workload_label(spec), "weights_per_gpu": n_w, "matrices": len(mc.slots), "streams": mc.n_streams,
                    "l2": "no flush: every phase streams 8.7-51 GB per step, far more than the 126 MB L2",
                    "step": "calibrate + encode + decode + distortion, phase by phase over all matrices",
                    "table": {"grid": int(mc.codebook.table_info()[0]), "bytes": int(mc.codebook.table_info()[5])},
@@ -308,7 +308,7 @@ def run_ours(args):
         "phases_ms": {"calibrate": cal_ms, "encode": enc_ms, "decode": dec_ms, "distortion": dis_ms},
         "clocks": clocks,
         "gpu_launches": mc.kernel_launches_per_step() * args.steps,
-        "roofline": {"kernel": "encode_kernel", "bound": "hbm", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
+        "roofline": {"kernel": "row_norm_kernel + encode_kernel (one qamw_encode call)", "bound": "hbm", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
                      "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": enc_gbs / 8000.0,
                      "algorithmic_bytes_per_launch": enc_bytes / n_launch, "avg_launch_ms": enc_ms / n_launch,
                      "traffic": None},
@@ -324,19 +324,32 @@ def run_ours(args):
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(spec, golden_or_trained_codebook(spec.K), args)
     traffic = load_traffic_note()
-    if traffic:
-        out["roofline"]["traffic"] = traffic.get("encode")
-        out["roofline_decode"]["traffic"] = traffic.get("decode")
+    if traffic:  # measured bytes per weight x weights of the average launch
+        out["roofline"]["traffic"] = traffic["encode"] * n_w / n_launch
+        out["roofline_decode"]["traffic"] = traffic["decode"] * n_w / n_launch
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
 def load_traffic_note():
-    """DRAM bytes per launch measured once with ncu (profiles/dram_traffic.json), if recorded."""
+    """DRAM bytes per weight measured once with ncu on the cfg4 matrix (profiles/dram_traffic.txt:
+    `key value` lines).  The note carries the hash of the kernel source it was taken from; if the
+    kernels have changed since, the traffic is unknown again (None)."""
+    import hashlib
     try:
-        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
-            return json.load(f)
+        note = {}
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for line in f:
+                if line.strip() and not line.startswith("#"):
+                    k, v = line.split()[:2]
+                    note[k] = v
+        src = os.path.join(ROOT, "paper_2605_26339_b200", "csrc", "qamw_kernels.cu")
+        with open(src, "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != note.get("kernel_source_sha256"):
+                return None
+        return {"encode": float(note["encode_dram_bytes_per_weight"]),
+                "decode": float(note["decode_dram_bytes_per_weight"])}
     except Exception:
         return None
 
