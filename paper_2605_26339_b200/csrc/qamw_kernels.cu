@@ -737,7 +737,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                 const int k0 = 4 * Layout<LOG2B_T>::octet_after(tid_g, rr);
                 if (k0 >= n_pairs) continue;
                 unsigned long long packed4 = 0ull;
-#pragma unroll 1
+#pragma unroll
                 for (int p = 0; p < 4; ++p) {
                     const float2 z = zst[(rr * 4 + p) * 32];
                     int v;
