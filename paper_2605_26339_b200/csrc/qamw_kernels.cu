@@ -154,11 +154,11 @@ __device__ __forceinline__ void bfly2(f32x2& a, f32x2& c) {
 // than 32, of the L threads of the block; stages in ascending order.  LOG2B_T >= 5: block size
 // 2^LOG2B_T known at compile time; LOG2B_T == 0: block size 2^log2b_rt <= 16 given at run time.
 // P[r][i] holds elements (2i, 2i+1) of the octet in slot r.
-template <int LOG2B_T>
+template <int LOG2B_T, bool FIRST_STAGE_DONE = false>
 __device__ __forceinline__ void fwht_regs(f32x2 (&P)[4][4], int log2b_rt, int tid_g) {
     typedef Layout<LOG2B_T> Lay;
     const int log2b = LOG2B_T ? LOG2B_T : log2b_rt;
-    if (log2b >= 1) {  // h = 1: inside a packed pair
+    if (log2b >= 1 && !FIRST_STAGE_DONE) {  // h = 1: inside a packed pair
 #pragma unroll
         for (int r = 0; r < 4; ++r)
 #pragma unroll
@@ -452,7 +452,11 @@ __device__ __forceinline__ float front_half(const RawRow<BF16>& raw, const f32x2
 // the copies of one entry fill consecutive 8-byte bank pairs and a lane that always reads copy
 // (lane mod C) only ever touches its own 16/C bank pairs.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void fill_codebook_copies(float2* dst, const float2* src, int K, int log2c) {
+// `butterfly`: store (x + y, x - y) instead of (x, y) -- the decoder's first butterfly stage works
+// on exactly these two numbers of every pair (scaled by the pair's sigma), so it can be done once
+// per codeword here instead of once per decoded pair.
+__device__ __forceinline__ void fill_codebook_copies(float2* dst, const float2* src, int K, int log2c,
+                                                     bool butterfly = false) {
     // all loads of a thread first (up to 8 in flight), then the copies as 16-byte stores
     constexpr int kMaxPerThread = 8;
     float2 c[kMaxPerThread];
@@ -462,6 +466,7 @@ __device__ __forceinline__ void fill_codebook_copies(float2* dst, const float2* 
         for (int u = 0; u < kMaxPerThread; ++u) {
             const int i = base + u * T + threadIdx.x;
             c[u] = i < K ? __ldg(src + i) : make_float2(0.f, 0.f);
+            if (butterfly) c[u] = make_float2(c[u].x + c[u].y, c[u].x - c[u].y);
         }
 #pragma unroll
         for (int u = 0; u < kMaxPerThread; ++u) {
@@ -1103,7 +1108,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
         }
         load8s(a.signs, e_out[r], g.d_in, g.cvec, sgn[r]);
     }
-    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
+    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c, true);
     f32x2 mcol[4][4];
 #pragma unroll
     for (int r = 0; r < 4; ++r)
@@ -1142,7 +1147,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
                 for (int p = 0; p < 4; ++p) P[r][p] = pack2(0.f, 0.f);
             }
         }
-        fwht_regs<LOG2B_T>(P, g.log2b, tid_g);
+        fwht_regs<LOG2B_T, true>(P, g.log2b, tid_g);  // stage h = 1 is already in the stored codewords
         const f32x2 rn2 = pack2(rn, rn);
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
