@@ -1,7 +1,7 @@
 """GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
 seeded inputs.
 
-Exactness rules (from the benchmark spec of this codec):
+Exactness rules of this codec:
   * packed indices bit-exact, except pairs whose oracle best / second-best squared distances
     differ by less than 1e-6 relative -- those are counted, and the GPU's choice must then be
     one of the two near-tied codewords;
