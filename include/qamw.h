@@ -55,6 +55,9 @@ extern "C" {
 #define QAMW_DTYPE_BF16 1
 
 #define QAMW_FLAG_BRUTE_FORCE 1u /* encode: exhaustive search over all K instead of the cell table */
+#define QAMW_FLAG_HALF_DEVICE 2u /* encode, decode, rotate: use every second SM only, so that two calls issued on
+                                    different streams run side by side and each one's start-up (tables and
+                                    per-column constants into shared memory and registers) hides behind the other */
 
 #define QAMW_DEFAULT_SIGN_SEED 0x51A5C0DEC0FFEE01ULL
 #define QAMW_MAX_BLOCK 1024 /* cap of Section 3.3 */

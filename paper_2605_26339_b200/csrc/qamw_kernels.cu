@@ -1337,6 +1337,12 @@ int sm_count() {
     return cached > 0 ? cached : 148;
 }
 
+// One persistent block per SM, or per second SM when the caller shares the device between two streams.
+int grid_limit(const qamw_params* p) {
+    const int n = sm_count();
+    return (p->flags & QAMW_FLAG_HALF_DEVICE) ? std::max(1, n / 2) : n;
+}
+
 int finish_launch(const char* what) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
@@ -1510,7 +1516,7 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     if (fixed + size_t(p->K) * 8 > kSmemLimit) return QAMW_ERR_NOMEM;
     a.log2c = pick_log2_copies(p->K, kSmemLimit - fixed);
     const size_t smem = fixed + (size_t(p->K) * 8 << a.log2c);
-    const int blocks = std::max(1, std::min(sm_count(), (p->d_out + a.g.groups - 1) / a.g.groups));
+    const int blocks = std::max(1, std::min(grid_limit(p), (p->d_out + a.g.groups - 1) / a.g.groups));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     {   // row norms first: the encoder proper reads them from row_norm_out
         NormArgs n;
@@ -1546,7 +1552,7 @@ extern "C" int qamw_rotate(const void* W, const qamw_params* p, const float* cha
     a.y_out = y_out;
     a.row_norm = row_norm_out;
     a.status = status_out;
-    const int blocks = std::max(1, std::min(sm_count(), (p->d_out + a.g.groups - 1) / a.g.groups));
+    const int blocks = std::max(1, std::min(grid_limit(p), (p->d_out + a.g.groups - 1) / a.g.groups));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define CALL(LB) rc = a.g.w_bf16 ? launch_aux<true, LB>(a, blocks, st) : launch_aux<false, LB>(a, blocks, st)
     QAMW_DISPATCH_LOG2B(a.g.log2b, CALL)
@@ -1695,7 +1701,7 @@ extern "C" int qamw_decode(const uint8_t* packed, const float* row_norm, const f
     const size_t stage_total = size_t(a.g.groups) * (a.g.tg / 32) * 2 * a.stage_bytes;
     a.log2c = pick_log2_copies(p->K, std::min(size_t(128) * 1024, kSmemLimit - stage_total));
     const size_t smem = (size_t(p->K) * 8 << a.log2c) + stage_total;
-    const int blocks = std::max(1, std::min(sm_count(), (p->d_out + a.g.groups - 1) / a.g.groups));
+    const int blocks = std::max(1, std::min(grid_limit(p), (p->d_out + a.g.groups - 1) / a.g.groups));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define CALL(LB) rc = launch_decode<LB>(a, blocks, smem, st)
     QAMW_DISPATCH_LOG2B(a.g.log2b, CALL)

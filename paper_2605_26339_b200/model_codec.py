@@ -86,7 +86,8 @@ class ModelCodec:
     def add_matrix(self, name: str, W: torch.Tensor, act_rms: torch.Tensor, sign_seed: int = q.DEFAULT_SIGN_SEED):
         spec, dev = self.spec, self.device
         d_out, d_in = W.shape
-        p = q.make_params(W, d_out, d_in, spec.block, spec.K)
+        # with several streams, consecutive matrices run side by side on half of the SMs each
+        p = q.make_params(W, d_out, d_in, spec.block, spec.K, q.FLAG_HALF_DEVICE if self.n_streams > 1 else 0)
         chan_scale = None
         if spec.alpha:
             chan_scale = torch.from_numpy(q.channel_scales(act_rms.cpu().numpy(), spec.alpha)).to(dev)
