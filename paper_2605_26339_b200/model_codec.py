@@ -86,8 +86,7 @@ class ModelCodec:
     def add_matrix(self, name: str, W: torch.Tensor, act_rms: torch.Tensor, sign_seed: int = q.DEFAULT_SIGN_SEED):
         spec, dev = self.spec, self.device
         d_out, d_in = W.shape
-        # with several streams, consecutive matrices run side by side on half of the SMs each
-        p = q.make_params(W, d_out, d_in, spec.block, spec.K, q.FLAG_HALF_DEVICE if self.n_streams > 1 else 0)
+        p = q.make_params(W, d_out, d_in, spec.block, spec.K)
         chan_scale = None
         if spec.alpha:
             chan_scale = torch.from_numpy(q.channel_scales(act_rms.cpu().numpy(), spec.alpha)).to(dev)
@@ -112,7 +111,10 @@ class ModelCodec:
 
     def _phase(self, call):
         cur = torch.cuda.current_stream(self.device)
-        if self.n_streams <= 1 or len(self.slots) <= 1:
+        side_by_side = self.n_streams > 1 and len(self.slots) > 1
+        for s in self.slots:  # consecutive matrices then run side by side on half of the SMs each
+            s.params.flags = (s.params.flags | q.FLAG_HALF_DEVICE) if side_by_side else (s.params.flags & ~q.FLAG_HALF_DEVICE)
+        if not side_by_side:
             for s in self.slots:
                 call(s, self.workspace, cur)
             return
