@@ -149,7 +149,7 @@ def oracle_pass(spec, probs, cb_host) -> float:
 
 def size_oracle_sample(spec, cb_host, seconds: float):
     """Probe with a few rows, then size the sample for about `seconds` of wall time."""
-    probe = oracle_sample_problem(spec, 32, 16, cb_host)
+    probe = oracle_sample_problem(spec, 256, 96, cb_host)
     oracle_pass(spec, probe, cb_host)  # first call builds / warms the library
     t = oracle_pass(spec, probe, cb_host)
     w = sum(p["rows"] * p["d_in"] for p in probe)
