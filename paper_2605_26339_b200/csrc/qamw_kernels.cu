@@ -143,6 +143,14 @@ struct Layout {
     }
 };
 
+// Ownership for kernels that do not rotate (row norms): slot r of lane l holds octet 32 r + l of the
+// warp's 128 octets, so every 16-byte load instruction of a warp covers 512 consecutive bytes.
+template <>
+struct Layout<-1> {
+    __device__ static __forceinline__ int octet_before(int tid_g, int r) { return 4 * (tid_g & ~31) + 32 * r + (tid_g & 31); }
+    __device__ static __forceinline__ int octet_after(int tid_g, int r) { return octet_before(tid_g, r); }
+};
+
 // (a, c) -> (a + c, a - c) on two packed registers.
 __device__ __forceinline__ void bfly2(f32x2& a, f32x2& c) {
     const f32x2 s = add2(a, c), d = sub2(a, c);
@@ -817,18 +825,18 @@ __global__ void __launch_bounds__(kMaxThreads, 1) row_norm_kernel(const NormArgs
     f32x2 t[4][4];
     {
         ColRaw craw;
-        load_col_raw<0>(craw, a.chan_scale, a.signs, g.d_in, g.cvec, tid_g);
+        load_col_raw<-1>(craw, a.chan_scale, a.signs, g.d_in, g.cvec, tid_g);
         col_factors(craw, t);
     }
     const long long row_step = (long long)gridDim.x * g.groups;
     long long row = (long long)blockIdx.x * g.groups + group;
     RawRow<BF16> raw;
-    if (row < g.d_out) load_row<BF16, 0>(raw, a.W, row, g, tid_g);
+    if (row < g.d_out) load_row<BF16, -1>(raw, a.W, row, g, tid_g);
     const int n_warps = g.tg >> 5;
     int parity = 0;
     for (; row < g.d_out; row += row_step, parity ^= 1) {
         RawRow<BF16> nxt;
-        if (row + row_step < g.d_out) load_row<BF16, 0>(nxt, a.W, row + row_step, g, tid_g);
+        if (row + row_step < g.d_out) load_row<BF16, -1>(nxt, a.W, row + row_step, g, tid_g);
         float x[4][8];
         raw_to_float<BF16>(raw, x);
         double ss = 0.0;

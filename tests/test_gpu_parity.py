@@ -305,6 +305,16 @@ def test_encode_decode_are_deterministic(orc):
     assert np.array_equal(a.what_full, b.what_full) and np.array_equal(a.sigma_gpu, b.sigma_gpu)
 
 
+def test_half_device_flag_changes_nothing_but_the_grid(orc):
+    """QAMW_FLAG_HALF_DEVICE only limits the number of blocks: same bits out, and parity still holds."""
+    W, act = _make(700, 2048, torch.bfloat16, 29)
+    a = Case(orc, W, act, 0.3, 128, 2048)
+    b = Case(orc, W, act, 0.3, 128, 2048, flags=q.FLAG_HALF_DEVICE)
+    b.check_all()
+    assert np.array_equal(a.packed, b.packed) and np.array_equal(a.norm, b.norm)
+    assert np.array_equal(a.what_full, b.what_full)
+
+
 def test_empty_matrix(orc):
     cb_host, cb = _codebook(orc, 64)
     p = q.make_params(None, 0, 64, 64, 64)
