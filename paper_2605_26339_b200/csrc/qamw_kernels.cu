@@ -1189,7 +1189,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
 // the tile and accumulates, per column, sum e^2 and sum w^2 over the rows of the chunk in double;
 // the activation weights r_j^2 are applied once per column at the end of the chunk.
 constexpr int kDistThreads = 128;
-constexpr int kDistRows = 32;
+constexpr int kDistRows = 16;
 
 template <bool BF16>
 __device__ __forceinline__ void dist_load(const void* W, long long w_row_stride, const __nv_bfloat16* What, int row,
@@ -1231,7 +1231,7 @@ __device__ __forceinline__ void dist_load(const void* W, long long w_row_stride,
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(kDistThreads, 6) distortion_kernel(const void* W, long long w_row_stride,
+__global__ void __launch_bounds__(kDistThreads, 5) distortion_kernel(const void* W, long long w_row_stride,
                                                                   const __nv_bfloat16* What, const float* act_rms,
                                                                   int d_out, int d_in, int vec, double* out4) {
     const int col_tiles = (d_in + 8 * kDistThreads - 1) / (8 * kDistThreads);
@@ -1247,7 +1247,47 @@ __global__ void __launch_bounds__(kDistThreads, 6) distortion_kernel(const void*
 #pragma unroll
         for (int e = 0; e < 8; ++e) E[e] = Q[e] = 0.0;
         int row = r0;
-        for (; row + 2 <= r1; row += 2) {  // two rows in flight per thread, eight blocks per SM
+        if (BF16 && vec) {
+            // bf16 fast path: the next two rows are loaded (as raw 16-byte words) before the current two
+            // are converted and accumulated, so four rows of loads are in flight per thread
+            auto ld = [&](int rw, uint4& wv, uint4& hv) {
+                const __nv_bfloat16* wrow = reinterpret_cast<const __nv_bfloat16*>(W) + (long long)rw * w_row_stride;
+                wv = __ldg(reinterpret_cast<const uint4*>(wrow + j0));
+                hv = __ldg(reinterpret_cast<const uint4*>(What + (long long)rw * d_in + j0));
+            };
+            auto acc = [&](const uint4& wv, const uint4& hv) {
+                const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w}, hw[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const double w0 = double(__uint_as_float(ww[i] << 16)), w1 = double(__uint_as_float(ww[i] & 0xffff0000u));
+                    const double d0 = w0 - double(__uint_as_float(hw[i] << 16));
+                    const double d1 = w1 - double(__uint_as_float(hw[i] & 0xffff0000u));
+                    E[2 * i] = fma(d0, d0, E[2 * i]);
+                    Q[2 * i] = fma(w0, w0, Q[2 * i]);
+                    E[2 * i + 1] = fma(d1, d1, E[2 * i + 1]);
+                    Q[2 * i + 1] = fma(w1, w1, Q[2 * i + 1]);
+                }
+            };
+            uint4 cw[2], ch[2], nw[2], nh[2];
+            if (row + 2 <= r1) {
+                ld(row, cw[0], ch[0]);
+                ld(row + 1, cw[1], ch[1]);
+            }
+            for (; row + 2 <= r1; row += 2) {
+                const bool more = row + 4 <= r1;
+                if (more) {
+                    ld(row + 2, nw[0], nh[0]);
+                    ld(row + 3, nw[1], nh[1]);
+                }
+                acc(cw[0], ch[0]);
+                acc(cw[1], ch[1]);
+                if (more) {
+                    cw[0] = nw[0]; ch[0] = nh[0];
+                    cw[1] = nw[1]; ch[1] = nh[1];
+                }
+            }
+        }
+        for (; row + 2 <= r1; row += 2) {  // generic path: two rows in flight per thread
             float w[2][8], h[2][8];
 #pragma unroll
             for (int u = 0; u < 2; ++u) dist_load<BF16>(W, w_row_stride, What, row + u, j0, d_in, vec, w[u], h[u]);
