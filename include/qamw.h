@@ -28,7 +28,7 @@
  *       h   = f32 butterfly of x per block, stages 1, 2, 4, ..., b/2, (a, b) -> (a+b, a-b);
  *       y_j = f32(h_j * g),  g = f32(c_b / r_i) (one f32 division),  c_b = f32(1 / sqrt((double)b));
  *       z   = f32(y * q_k),  q_k = f32(1 / (double)sigma_k);
- *       idx = argmin_c fma(dy, dy, dx*dx) in f32 with dx = z_x - c_x, dy = z_y - c_y,
+ *       idx = argmin_c f32(f32(dx*dx) + f32(dy*dy)) with dx = f32(z_x - c_x), dy = f32(z_y - c_y),
  *             lowest index among equal distances.
  *     A row with r_i == 0 is encoded as the origin's codeword in every pair and decodes to zeros.
  *     A row whose norm is not finite sets bit 0 of *status_out; its indices are unspecified.

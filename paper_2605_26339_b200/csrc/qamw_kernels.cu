@@ -534,10 +534,13 @@ __device__ __forceinline__ float2 codeword(const SearchSmem& s, int k) {
     return lds_f32x2(s.cb + (uint32_t(k) << s.cb_shift));
 }
 
-// Squared distance in direct form, one rounding per operation: (zx-cx)^2 + (zy-cy)^2.
+// Squared distance in direct form, one rounding per operation: f32(f32(dx^2) + f32(dy^2)); the two
+// subtractions and the two squares are one packed instruction each.
 __device__ __forceinline__ float dist2(float2 c, float zx, float zy) {
-    const float dx = __fsub_rn(zx, c.x), dy = __fsub_rn(zy, c.y);
-    return __fmaf_rn(dy, dy, __fmul_rn(dx, dx));
+    const f32x2 d = sub2(pack2(zx, zy), pack2(c.x, c.y));
+    float sx, sy;
+    unpack2(mul2(d, d), sx, sy);
+    return __fadd_rn(sx, sy);
 }
 
 __device__ __forceinline__ void consider(const SearchSmem& s, int k, float zx, float zy, float& best, int& arg) {
