@@ -22,6 +22,12 @@
 //   * Shared-memory reads are what limits these kernels on B200 (random 8-byte reads replay on
 //     bank conflicts), hence: the codebook is stored in several bank-separated copies and every
 //     lane reads the copy of its own banks.
+//   * A warp owns 1024 consecutive elements: whole Hadamard blocks and 64*B consecutive bytes of
+//     the packed row.  The encoder (whose row norms come from a kernel of their own) and the
+//     decoder therefore have no barrier after their prologue; each warp stages its own piece of
+//     the packed row in shared memory.
+//   * The encoder's search exists once in its instruction stream (a rolled loop fed from a
+//     lane-private staging area): sixteen inlined copies per row overflow the instruction cache.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
