@@ -367,7 +367,7 @@ def run_e2e(mc, args, world, dist):
     n_layers = len(slots) // per_layer
     layer_bytes = sum(s.W.numel() * s.W.element_size() for s in slots[:per_layer])
     avail = psutil.virtual_memory().available
-    host_layers = max(1, min(n_layers, int(0.35 * avail / layer_bytes)))
+    host_layers = max(1, min(n_layers, int(0.35 * avail / max(1, world) / layer_bytes)))  # all ranks share the host
     host_W = []
     for s in slots[: host_layers * per_layer]:
         h = torch.empty(s.W.shape, dtype=s.W.dtype, pin_memory=True)
