@@ -58,6 +58,7 @@ constexpr int kMaxThreads = 512;   // threads per block (register budget: 128 pe
 constexpr int kMaxGroups = 15;     // named barriers 1..15
 constexpr unsigned kFull = 0xffffffffu;
 constexpr size_t kSmemLimit = 227 * 1024;
+constexpr size_t kEncodeStaticSmem = 512;  // the encoder's statically allocated partial sums
 
 struct RowGeom {
     int d_out, d_in;
@@ -147,14 +148,6 @@ struct Layout {
         const int hi = (S & 1) ? (((r >> 1) & 1) | ((r & 1) << 1)) : r;
         return blk * (4 * L) + q + L * hi;
     }
-};
-
-// Ownership for kernels that do not rotate (row norms): slot r of lane l holds octet 32 r + l of the
-// warp's 128 octets, so every 16-byte load instruction of a warp covers 512 consecutive bytes.
-template <>
-struct Layout<-1> {
-    __device__ static __forceinline__ int octet_before(int tid_g, int r) { return 4 * (tid_g & ~31) + 32 * r + (tid_g & 31); }
-    __device__ static __forceinline__ int octet_after(int tid_g, int r) { return octet_before(tid_g, r); }
 };
 
 // (a, c) -> (a + c, a - c) on two packed registers.
@@ -628,20 +621,23 @@ struct EncodeArgs {
     long long packed_row_stride;  // bytes
     int row_words;           // 32-bit words per packed row (stride / 4)
     int payload_words;       // words that hold index bits: ceil(row payload bytes / 4)
-    const float* row_norm;   // written by row_norm_kernel just before
+    float* row_norm;         // out: r_i
+    int32_t* status;         // out (optional): bit 0 set when a row norm is not finite
 };
 
 constexpr int kStageSlotsPerWarp = 128 + 4 * 8;  // 128 octets of a warp plus their padding
 
-// Encoder proper.  The row norms are already in global memory, so the warps of a row share
-// nothing: a warp owns 1024 consecutive elements (whole Hadamard blocks), rotates them with
-// shuffles, searches its 512 pairs, stages the indices in its own piece of shared memory and
-// writes its 64*B bytes of the packed row.  No block-wide barrier after the prologue.
+// Encoder.  A warp owns 1024 consecutive elements of a row (whole Hadamard blocks): it rotates
+// them with shuffles, searches its 512 pairs, stages the indices in its own piece of shared
+// memory and writes its 64*B bytes of the packed row.  The warps of a row share one thing, the
+// row norm: each adds its partial sum of squares to shared memory and they meet at one named
+// barrier per row, after the rotation.  W is read once.
 template <bool BF16, int LOG2B_T>
 __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ double ss_part[2][32];  // per-warp partial sums of squares, two rows in flight
     const RowGeom& g = a.g;
-    // shared memory: [codebook copies][table][index staging: one piece per warp]
+    // dynamic shared memory: [codebook copies][table][index staging: one piece per warp]
     const int group = threadIdx.x / g.tg;
     const int tid_g = threadIdx.x - group * g.tg;
     const int lane = threadIdx.x & 31;
@@ -718,20 +714,17 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     const int oct0 = 128 * warp_g;                 // its first octet
     const int seg_word0 = 16 * B * warp_g;         // its first packed word (64*B bytes per segment)
     const bool last_seg = (warp_g + 1) * 1024 >= g.d_in;
+    const int n_warps = g.tg >> 5;
 
     // The row loop exists in three variants chosen once per block, so that the common one carries
     // no call to the rarely needed searches: 0 = table search, 1 = table search with the reach
     // check, 2 = exhaustive search.
     auto rows = [&](auto mode_tag) {
         constexpr int MODE = decltype(mode_tag)::value;
-        for (long long row = (long long)blockIdx.x * g.groups + group; row < g.d_out; row += row_step) {
+        int parity = 0;
+        for (long long row = (long long)blockIdx.x * g.groups + group; row < g.d_out; row += row_step, parity ^= 1) {
             RawRow<BF16> raw;
             load_row<BF16, LOG2B_T>(raw, a.W, row, g, tid_g);
-            const float r = __ldg(a.row_norm + row);
-            // g = f32(c_b / r); 0 for a zero row (all its pairs become the origin, 0 * 0) and for a
-            // non-finite row (its indices are unspecified; the searches accept any input)
-            const float gn = (isfinite(r) && r > 0.f) ? __fdiv_rn(a.inv_sqrt_b, r) : 0.f;
-            const f32x2 gn2 = pack2(gn, gn);
             f32x2 P[4][4];
             {
                 float x[4][8];
@@ -741,7 +734,42 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
 #pragma unroll
                     for (int i = 0; i < 4; ++i) P[rr][i] = mul2(pack2(x[rr][2 * i], x[rr][2 * i + 1]), t[rr][i]);
             }
+            // sum of squares of the row: ss = sum_j (double)x_j^2, per thread, per warp, then per row
+            double* part = &ss_part[parity][threadIdx.x >> 5] - warp_g;  // the row's per-warp sums
+            {
+                double ss = 0.0;
+#pragma unroll
+                for (int rr = 0; rr < 4; ++rr)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        float p, c;
+                        unpack2(P[rr][i], p, c);
+                        const double pd = double(p), cd = double(c);
+                        ss = fma(pd, pd, ss);
+                        ss = fma(cd, cd, ss);
+                    }
+                ss = warp_sum(ss);
+                if (lane == 0) part[warp_g] = ss;
+            }
+            // The rotation does not need the norm, so the warps of the row meet only after it.  A
+            // warp can be one row ahead of another at most, hence the two sets of partial sums.
             fwht_regs<LOG2B_T>(P, g.log2b, tid_g);
+            group_barrier(group, g.tg);
+            float gn = 0.f;
+            if (lane == 0) {  // every warp adds the same numbers in the same order
+                double total = 0.0;
+                for (int w = 0; w < n_warps; ++w) total += part[w];
+                const float r = float(sqrt(total));
+                // g = f32(c_b / r); 0 for a zero row (all its pairs become the origin, 0 * 0) and for a
+                // non-finite row (its indices are unspecified; the searches accept any input)
+                if (isfinite(r) && r > 0.f) gn = __fdiv_rn(a.inv_sqrt_b, r);
+                if (warp_g == 0) {
+                    a.row_norm[row] = r;
+                    if (!isfinite(r) && a.status) atomicOr(a.status, 1);
+                }
+            }
+            gn = __shfl_sync(kFull, gn, 0);
+            const f32x2 gn2 = pack2(gn, gn);
             // The sixteen points of the thread go through a lane-private piece of shared memory, so
             // that the search exists once in the instruction stream: a fully unrolled row loop does
             // not fit the instruction cache, and fetch stalls then cost more than the extra
@@ -806,72 +834,6 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     if (a.brute) rows(std::integral_constant<int, 2>{});
     else if (any_risky) rows(std::integral_constant<int, 1>{});
     else rows(std::integral_constant<int, 0>{});
-}
-
-// ---------------------------------------------------------------------------------------------
-// row-norm kernel: r_i = f32(sqrt(sum_j (double)x_ij^2)), x_ij = f32(W_ij * t_j)
-// ---------------------------------------------------------------------------------------------
-// Same thread geometry as the other row kernels (a thread owns 32 columns, its factors t stay in
-// registers, the next row is prefetched into registers).  The warps of a row meet at one barrier
-// per row; nobody waits for the result, which goes to global memory for the encoder proper.
-
-struct NormArgs {
-    RowGeom g;
-    const void* W;
-    const float* chan_scale;
-    const int8_t* signs;
-    float* row_norm;
-    int32_t* status;
-};
-
-template <bool BF16>
-__global__ void __launch_bounds__(kMaxThreads, 1) row_norm_kernel(const NormArgs a) {
-    __shared__ double red_all[kMaxGroups * 64];
-    const RowGeom& g = a.g;
-    const int group = threadIdx.x / g.tg;
-    const int tid_g = threadIdx.x - group * g.tg;
-    double* red = red_all + group * 64;
-    f32x2 t[4][4];
-    {
-        ColRaw craw;
-        load_col_raw<-1>(craw, a.chan_scale, a.signs, g.d_in, g.cvec, tid_g);
-        col_factors(craw, t);
-    }
-    const long long row_step = (long long)gridDim.x * g.groups;
-    long long row = (long long)blockIdx.x * g.groups + group;
-    RawRow<BF16> raw;
-    if (row < g.d_out) load_row<BF16, -1>(raw, a.W, row, g, tid_g);
-    const int n_warps = g.tg >> 5;
-    int parity = 0;
-    for (; row < g.d_out; row += row_step, parity ^= 1) {
-        RawRow<BF16> nxt;
-        if (row + row_step < g.d_out) load_row<BF16, -1>(nxt, a.W, row + row_step, g, tid_g);
-        float x[4][8];
-        raw_to_float<BF16>(raw, x);
-        double ss = 0.0;
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float p, c;
-                unpack2(mul2(pack2(x[r][2 * i], x[r][2 * i + 1]), t[r][i]), p, c);
-                const double pd = double(p), cd = double(c);
-                ss = fma(pd, pd, ss);
-                ss = fma(cd, cd, ss);
-            }
-        ss = warp_sum(ss);
-        double* slot = red + parity * 32;
-        if ((tid_g & 31) == 0) slot[tid_g >> 5] = ss;
-        group_barrier(group, g.tg);
-        if (tid_g == 0) {
-            double total = 0.0;
-            for (int w = 0; w < n_warps; ++w) total += slot[w];
-            const float r = float(sqrt(total));
-            a.row_norm[row] = r;
-            if (!isfinite(r) && a.status) atomicOr(a.status, 1);
-        }
-        raw = nxt;
-    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1437,12 +1399,6 @@ int launch_encode(const EncodeArgs& a, int blocks, size_t smem, cudaStream_t st)
     return finish_launch("encode_kernel");
 }
 
-template <bool BF16>
-int launch_norm(const NormArgs& a, int blocks, cudaStream_t st) {
-    row_norm_kernel<BF16><<<blocks, a.g.tg * a.g.groups, 0, st>>>(a);
-    return finish_launch("row_norm_kernel");
-}
-
 template <bool BF16, int LOG2B_T>
 int launch_aux(const AuxArgs& a, int blocks, cudaStream_t st) {
     aux_kernel<BF16, LOG2B_T><<<blocks, a.g.tg * a.g.groups, 0, st>>>(a);
@@ -1486,7 +1442,7 @@ extern "C" int qamw_codebook_create(const float* codebook_host, int K, int grid,
     // indices + 4 KB of points)) and the codebook in four bank-separated copies (one copy for
     // K = 4096): the table gets what is left of the 227 KB of one SM.
     const size_t copies = K <= 2048 ? 4 : 1;
-    const size_t budget = kSmemLimit - size_t(16) * (kStageSlotsPerWarp * 8 + 512 * 8) - size_t(K) * 8 * copies;
+    const size_t budget = kSmemLimit - kEncodeStaticSmem - size_t(16) * (kStageSlotsPerWarp * 8 + 512 * 8) - size_t(K) * 8 * copies;
     if (!choose_search_table(codebook_host, K, grid, budget, &t)) return QAMW_ERR_NOMEM;
     qamw_codebook* cb = new (std::nothrow) qamw_codebook();
     if (!cb) return QAMW_ERR_NOMEM;
@@ -1570,22 +1526,12 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     a.inv_sqrt_b = float(1.0 / std::sqrt(double(p->block)));
     const size_t fixed = ((size_t(a.table_bytes) + 15) & ~size_t(15)) +
                          size_t(a.g.groups) * (a.g.tg / 32) * (kStageSlotsPerWarp * 8 + 512 * 8);
-    if (fixed + size_t(p->K) * 8 > kSmemLimit) return QAMW_ERR_NOMEM;
-    a.log2c = pick_log2_copies(p->K, kSmemLimit - fixed);
+    if (fixed + size_t(p->K) * 8 > kSmemLimit - kEncodeStaticSmem) return QAMW_ERR_NOMEM;
+    a.log2c = pick_log2_copies(p->K, kSmemLimit - kEncodeStaticSmem - fixed);
     const size_t smem = fixed + (size_t(p->K) * 8 << a.log2c);
     const int blocks = std::max(1, std::min(grid_limit(p), (p->d_out + a.g.groups - 1) / a.g.groups));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    {   // row norms first: the encoder proper reads them from row_norm_out
-        NormArgs n;
-        n.g = a.g;
-        n.W = W;
-        n.chan_scale = chan_scale;
-        n.signs = signs;
-        n.row_norm = row_norm_out;
-        n.status = status_out;
-        rc = a.g.w_bf16 ? launch_norm<true>(n, blocks, st) : launch_norm<false>(n, blocks, st);
-        if (rc) return rc;
-    }
+    a.status = status_out;
 #define CALL(LB)                                                                  \
     rc = a.g.w_bf16 ? launch_encode<true, LB>(a, blocks, smem, st) : launch_encode<false, LB>(a, blocks, smem, st)
     QAMW_DISPATCH_LOG2B(a.g.log2b, CALL)

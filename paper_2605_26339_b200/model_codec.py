@@ -167,9 +167,8 @@ class ModelCodec:
         return enc, dec
 
     def kernel_launches_per_step(self) -> int:
-        # calibrate = 2 kernels, encode = 2 (row norms, encoder), decode 1, distortion 1 (its memset is
-        # not a kernel of ours)
-        return 6 * len(self.slots)
+        # calibrate = 2 kernels, encode 1, decode 1, distortion 1 (its memset is not a kernel of ours)
+        return 5 * len(self.slots)
 
     def totals(self, group=None) -> Dict[str, float]:
         """Error figures over all matrices of all ranks (see combine_distortion)."""
