@@ -121,10 +121,12 @@ int qamw_status_to_error(int32_t status_word);
 
 /* Uploads the K x 2 f32 codebook (host pointer) to the current device and builds the exact
  * spatial search table used by qamw_encode (Section 3.6: "nearest codebook entry by Euclidean
- * distance"): [-8, 8)^2 is cut into grid x grid cells whose boundaries follow the quantiles of
- * N(0, 2); every cell lists all codewords whose nearest-neighbour region can meet the cell, so a
- * scan of the list returns what a scan of the whole codebook returns.  Points outside [-8, 8)^2
- * are scanned exhaustively.  grid = 0 picks a default (about 2.1 sqrt(K)).  Synchronous.
+ * distance"): the plane is cut into grid x grid cells, narrow where a Gaussian source puts its
+ * codewords and widening outwards; every cell lists all codewords whose nearest-neighbour region
+ * can meet the cell, so a scan of the list returns what a scan of the whole codebook returns.
+ * The outermost cells reach to |z| < 16384; points beyond are scanned exhaustively.  grid = 0
+ * picks a default (about 2.2 sqrt(K)); an explicit grid must be odd and at most 255, else
+ * QAMW_ERR_ARG.  Synchronous.
  * *out must be released with qamw_codebook_destroy on the same device. */
 int qamw_codebook_create(const float* codebook_host, int K, int grid, qamw_codebook** out);
 void qamw_codebook_destroy(qamw_codebook* cb);
@@ -133,13 +135,17 @@ void qamw_codebook_destroy(qamw_codebook* cb);
  * candidate list, number of cells with more than four candidates, overflow entries, table bytes. */
 int qamw_codebook_table_info(const qamw_codebook* cb, int32_t* info_out);
 
-/* Host-only construction of the same table, for inspection and tests (no CUDA).  lut_out: 4096
- * bytes mapping fine bin floor(z*256 + 2048) to a grid column/row; cells_out: grid*grid records of
- * four u16 (ascending candidate indices, last repeated as padding; or {0xFFFF, offset, count, 0}
- * pointing into overflow_out).  Any output pointer may be NULL; info_out as above (6 values).
+/* Host-only construction of the same table, for inspection and tests (no CUDA).  map_out: four
+ * floats {zmax, c0, c1, c2} of the map from a coordinate to its column (and, alike, its row):
+ *     c = min(max(z, -zmax), zmax), t = c * c, column = (grid - 1) / 2 + rn(c (c0 + t (c1 + t c2)))
+ * which the device evaluates in f32 with fused multiply-adds; a point within 2^-8 of a column
+ * boundary (in units of columns) is covered by the lists of both neighbours.  cells_out:
+ * grid*grid records of four u16, row-major (ascending candidate indices, last repeated as
+ * padding; or {0xFFFF, offset, count, 0} pointing into overflow_out).  Any output pointer may
+ * be NULL; info_out as above (6 values).
  * Returns QAMW_ERR_NOMEM if the table does not fit budget_bytes or a capacity. */
 int qamw_search_table_build(const float* codebook_host, int K, int grid, size_t budget_bytes,
-                            uint8_t* lut_out, uint16_t* cells_out, size_t cells_cap,
+                            float* map_out, uint16_t* cells_out, size_t cells_cap,
                             uint16_t* overflow_out, size_t overflow_cap, int32_t* info_out);
 
 /* ----------------------------------------------------------------------------------------------

@@ -146,20 +146,21 @@ def status_to_error(status_word: int) -> int:
 
 
 def search_table_build(codebook, grid: int = 0, budget_bytes: int = 1 << 20):
-    """Host-only table construction -> (lut u8[4096], cells u16[grid*grid,4], overflow u16[], info[6])."""
+    """Host-only table construction -> (map f32[4] = zmax, c0, c1, c2; cells u16[grid*grid,4]; overflow u16[];
+    info[6])."""
     cb = _np(codebook, np.float32)
     K = cb.shape[0]
     info = np.zeros(6, np.int32)
     _check("qamw_search_table_build", lib().qamw_search_table_build(cb.ctypes.data, K, grid, budget_bytes, None,
                                                                     None, 0, None, 0, info.ctypes.data))
     g = int(info[0])
-    lut = np.zeros(4096, np.uint8)
+    cmap = np.zeros(4, np.float32)
     cells = np.zeros((g * g, 4), np.uint16)
     ovf = np.zeros(max(1, int(info[4])), np.uint16)
     _check("qamw_search_table_build", lib().qamw_search_table_build(cb.ctypes.data, K, g, budget_bytes,
-                                                                    lut.ctypes.data, cells.ctypes.data, cells.size,
+                                                                    cmap.ctypes.data, cells.ctypes.data, cells.size,
                                                                     ovf.ctypes.data, ovf.size, info.ctypes.data))
-    return lut, cells, ovf, info
+    return cmap, cells, ovf, info
 
 
 # ------------------------------------------------------------------------------- codebook object

@@ -67,8 +67,12 @@ constexpr int kChunks = 64;
 double assign_pass(const std::vector<double>& samples, uint64_t n, const std::vector<double>& cb, int K,
                    std::vector<double>* sums /* kChunks*K*2 or null */, std::vector<int64_t>* counts /* kChunks*K */) {
     CellLists cells;
-    int grid = std::max(2, default_grid(K) / 2);
+    int grid = std::max(3, (default_grid(K) / 4) * 2 + 1);
     bool ok = build_cell_lists(cb.data(), K, grid, &cells);
+    auto column_of = [&](double z) {  // a point near a boundary may get either neighbour: both lists hold its answer
+        const int c = cells.map.half + int(std::lround(cell_map_value(cells.map, z)));
+        return size_t(std::min(grid - 1, std::max(0, c)));
+    };
     std::vector<double> chunk_err(kChunks, 0.0);
     if (sums) std::fill(sums->begin(), sums->end(), 0.0);
     if (counts) std::fill(counts->begin(), counts->end(), int64_t(0));
@@ -79,7 +83,6 @@ double assign_pass(const std::vector<double>& samples, uint64_t n, const std::ve
         int64_t* cnt = counts ? counts->data() + size_t(c) * K : nullptr;
         for (uint64_t i = lo; i < hi; ++i) {
             double zx = samples[2 * i], zy = samples[2 * i + 1];
-            double fx = std::floor(zx * kFineScale + kFineOffset), fy = std::floor(zy * kFineScale + kFineOffset);
             double best = INFINITY;
             int arg = 0;
             auto consider = [&](int k) {
@@ -91,9 +94,7 @@ double assign_pass(const std::vector<double>& samples, uint64_t n, const std::ve
                 }
             };
             if (ok && std::fabs(zx) < 16000.0 && std::fabs(zy) < 16000.0) {
-                const size_t bx = size_t(std::min(double(kFineBins - 1), std::max(0.0, fx)));
-                const size_t by = size_t(std::min(double(kFineBins - 1), std::max(0.0, fy)));
-                const auto& list = cells.lists[size_t(cells.lut[by]) * grid + cells.lut[bx]];
+                const auto& list = cells.lists[column_of(zy) * grid + column_of(zx)];
                 for (uint16_t k : list) consider(int(k));
             } else {
                 for (int k = 0; k < K; ++k) consider(k);

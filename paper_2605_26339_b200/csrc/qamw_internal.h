@@ -16,16 +16,27 @@ inline int ilog2(int64_t v) {
     return l;
 }
 
-// Fine binning of one axis: bin = clamp(floor(z * kFineScale + kFineOffset), 0, kFineBins - 1).
-constexpr int kFineBins = 4096;
-constexpr double kFineScale = 256.0;
-constexpr double kFineOffset = 2048.0;
+// Column (and, with the same map, row) of the search grid that holds coordinate z:
+//     c = min(max(z, -zmax), zmax);  t = c * c;
+//     column = half + rn(c * (c0 + t * (c1 + t * c2)))            (rn: to nearest integer)
+// an odd polynomial whose slope falls like (1 - t / T)^2: cells are narrow where a Gaussian source
+// puts its codewords and widen towards zmax; the outermost columns take everything beyond.  The
+// device evaluates it in f32 (three fused multiply-adds, the last one onto 1.5 * 2^23 + half, which
+// leaves the integer in the low mantissa bits).  grid = 2 * half + 1 is odd.
+struct CellMap {
+    int grid = 0, half = 0;
+    float zmax = 0.f, c0 = 0.f, c1 = 0.f, c2 = 0.f;
+};
+CellMap make_cell_map(int grid);
+// The map in exact arithmetic on the f32 coefficients (before rounding to an integer).
+double cell_map_value(const CellMap& m, double z);
 
-// Host form of the search grid: per coarse cell the full candidate list.
+// Host form of the search grid: per cell the full candidate list.
 struct CellLists {
-    int grid = 0;
-    std::vector<double> edges;        // grid+1 coarse boundaries (z units); the outermost are +-16384
-    std::vector<uint8_t> lut;         // fine bin -> coarse column / row
+    CellMap map;
+    // Column j can be returned by the device for z in [lo[j], hi[j]]: the interval of the exact map
+    // widened by a margin that covers the device's rounding; the outermost reach +-16384.
+    std::vector<double> lo, hi;
     std::vector<std::vector<uint16_t>> lists;  // [iy*grid + ix], ascending codeword indices
     int max_list = 0;
     int n_candidates = 0;
@@ -33,21 +44,20 @@ struct CellLists {
 
 // Device form (see pack_search_table in qamw_table.cpp).
 struct SearchTable {
-    int grid = 0;
-    std::vector<uint8_t> lut;         // kFineBins bytes
+    CellMap map;
     std::vector<uint16_t> cells;      // grid*grid records of 4 x u16
     std::vector<uint16_t> overflow;   // candidate lists of cells with more than 4 entries
     int n_overflow_cells = 0;
     int max_list = 0;
     int n_candidates = 0;
-    size_t bytes() const { return lut.size() + cells.size() * 2 + overflow.size() * 2; }
+    size_t bytes() const { return cells.size() * 2 + overflow.size() * 2; }
 };
 
 int default_grid(int K);
 bool build_cell_lists(const double* cb, int K, int grid, CellLists* out);
 bool pack_search_table(const CellLists& cl, SearchTable* out);
 
-// grid > 0: exactly that grid (fails if it does not fit); grid == 0: the default grid for K,
+// grid > 0 (odd): exactly that grid (fails if it does not fit); grid == 0: the default grid for K,
 // shrunk until the table fits in budget_bytes.
 bool choose_search_table(const float* codebook, int K, int grid, size_t budget_bytes, SearchTable* out);
 
@@ -58,11 +68,11 @@ void set_cuda_error(const char* what, int code);
 struct qamw_codebook {
     int K = 0;
     int device = -1;
-    // one device allocation: [codebook K*2 f32][cells grid^2 * 4 u16][overflow u16][lut 4096 u8]
+    // one device allocation: [codebook K*2 f32][cells grid^2 * 4 u16][overflow u16]
     void* d_blob = nullptr;
     size_t blob_bytes = 0;
-    size_t off_cells = 0, off_overflow = 0, off_lut = 0;
-    int grid = 0;
+    size_t off_cells = 0, off_overflow = 0;
+    qamw::CellMap map;
     int n_candidates = 0, max_list = 0, n_overflow_cells = 0;
     std::vector<float> h_codebook;  // host copy (decode only needs the device codebook)
 };

@@ -508,11 +508,6 @@ __device__ __forceinline__ uint2 lds_u32x2(uint32_t addr) {
     asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
-    uint32_t v;
-    asm("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
 __device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
     uint32_t v;
     asm("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));
@@ -522,12 +517,16 @@ __device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
 struct SearchSmem {       // all fields are shared-memory byte addresses
     uint32_t cb;          // codebook copies, already offset to this lane's copy
     int cb_shift;         // log2 of the byte distance between consecutive entries (3 + log2c)
-    uint32_t cells;       // grid*grid records of 8 bytes
+    uint32_t cells;       // grid*grid records of 8 bytes; minus 8 * (grid + 1) * kMagicBits, see search_cell
     uint32_t overflow;    // u16 lists
-    uint32_t lut;         // 4096 bytes
-    int grid;
+    uint32_t grid;
     int K;
+    f32x2 zlo;            // the cell map, each value twice: -zmax,
+    f32x2 c0, c1, c2;     // the polynomial's coefficients,
+    f32x2 bias;           // 1.5 * 2^23 + half
 };
+
+constexpr uint32_t kMagicBits = 0x4B400000u;  // bit pattern of 1.5 * 2^23 = 12582912.0f
 
 __device__ __forceinline__ float2 codeword(const SearchSmem& s, int k) {
     return lds_f32x2(s.cb + (uint32_t(k) << s.cb_shift));
@@ -566,13 +565,23 @@ __device__ __forceinline__ int search_overflow(const SearchSmem& s, uint2 rec, f
     return arg;
 }
 
-// Table search for a point known to lie inside the table's reach (|z| < 16000, not NaN).
+// Table search for a point known to lie inside the table's reach (|z| < 16000; a NaN coordinate
+// is clamped like a large one and gets some index).
 __device__ __forceinline__ int search_cell(const SearchSmem& s, float zx, float zy) {
-    // fine bin = clamp(floor(z * 256 + 2048), 0, 4095); the conversion saturates negatives to 0
-    const unsigned bx = min(__float2uint_rz(__fmaf_rn(zx, 256.0f, 2048.0f)), 4095u);
-    const unsigned by = min(__float2uint_rz(__fmaf_rn(zy, 256.0f, 2048.0f)), 4095u);
-    const uint32_t ix = lds_u8(s.lut + bx), iy = lds_u8(s.lut + by);
-    const uint2 rec = lds_u32x2(s.cells + 8u * (iy * uint32_t(s.grid) + ix));
+    // Column and row: c = clamp(z, +-zmax), half + rn(c (c0 + t (c1 + t c2))), t = c^2, both axes in
+    // packed arithmetic.  The last fused multiply-add lands on 1.5 * 2^23 + half, where the spacing
+    // of f32 is 1: its rounding is the rounding to an integer, and the integer sits in the low
+    // mantissa bits, kMagicBits above zero.  That offset is folded into s.cells.
+    float lo, hi;
+    unpack2(s.zlo, lo, hi);
+    const float cx = fminf(fmaxf(zx, lo), -lo), cy = fminf(fmaxf(zy, lo), -lo);
+    const f32x2 c = pack2(cx, cy);
+    const f32x2 t = mul2(c, c);
+    const f32x2 v = fma2(c, fma2(t, fma2(t, s.c2, s.c1), s.c0), s.bias);
+    float vx, vy;
+    unpack2(v, vx, vy);
+    const uint32_t bx = __float_as_uint(vx), by = __float_as_uint(vy);
+    const uint2 rec = lds_u32x2(s.cells + ((by * s.grid + bx) << 3));
     const int k0 = int(rec.x & 0xffffu);
     if (k0 == 0xffff) return search_overflow(s, rec, zx, zy);
     const int k1 = int(rec.x >> 16), k2 = int(rec.y & 0xffffu), k3 = int(rec.y >> 16);
@@ -610,10 +619,11 @@ struct EncodeArgs {
     const int8_t* signs;
     const float* sigma;
     const float2* codebook;  // device, K entries
-    const uint4* table;      // cells | overflow | lut, as laid out by qamw_codebook_create
-    int table_bytes;
-    int off_overflow, off_lut;  // byte offsets inside the table
+    const uint4* table;      // cells | overflow, as laid out by qamw_codebook_create
+    int table_bytes;         // a multiple of 16
+    int off_overflow;        // byte offset inside the table
     int K, log2K, grid;
+    float map_zmax, map_c0, map_c1, map_c2, map_bias;  // the cell map of the table
     int log2c;               // log2 of the number of codebook copies in shared memory
     int brute;
     float inv_sqrt_b;        // c_b = f32(1 / sqrt(b))
@@ -700,11 +710,15 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     SearchSmem s;
     s.cb = smem_addr(smem) + 8u * (threadIdx.x & ((1 << a.log2c) - 1));
     s.cb_shift = 3 + a.log2c;
-    s.cells = smem_addr(table);
+    s.cells = smem_addr(table) - 8u * kMagicBits * uint32_t(a.grid + 1);
     s.overflow = smem_addr(table + a.off_overflow);
-    s.lut = smem_addr(table + a.off_lut);
-    s.grid = a.grid;
+    s.grid = uint32_t(a.grid);
     s.K = a.K;
+    s.zlo = pack2(-a.map_zmax, -a.map_zmax);
+    s.c0 = pack2(a.map_c0, a.map_c0);
+    s.c1 = pack2(a.map_c1, a.map_c1);
+    s.c2 = pack2(a.map_c2, a.map_c2);
+    s.bias = pack2(a.map_bias, a.map_bias);
 
     const long long row_step = (long long)gridDim.x * g.groups;
     const int B = a.log2K, B4 = 4 * a.log2K;
@@ -1435,32 +1449,30 @@ extern "C" const char* qamw_last_cuda_error(void) { return g_last_error; }
 extern "C" int qamw_codebook_create(const float* codebook_host, int K, int grid, qamw_codebook** out) {
     if (!codebook_host || !out) return QAMW_ERR_ARG;
     if (K < 2 || K > QAMW_MAX_K || !is_pow2(K)) return QAMW_ERR_SHAPE;
-    if (grid < 0 || grid > 255) return QAMW_ERR_ARG;
+    if (grid < 0 || grid > 255 || (grid > 0 && grid % 2 == 0)) return QAMW_ERR_ARG;
     *out = nullptr;
     SearchTable t;
     // The encoder's shared memory also holds 84 KB of per-warp staging (16 warps x (1.25 KB of
     // indices + 4 KB of points)) and the codebook in four bank-separated copies (one copy for
-    // K = 4096): the table gets what is left of the 227 KB of one SM.
+    // K = 4096): the table gets what is left of the 227 KB of one SM.  The grid side is odd.
     const size_t copies = K <= 2048 ? 4 : 1;
     const size_t budget = kSmemLimit - kEncodeStaticSmem - size_t(16) * (kStageSlotsPerWarp * 8 + 512 * 8) - size_t(K) * 8 * copies;
     if (!choose_search_table(codebook_host, K, grid, budget, &t)) return QAMW_ERR_NOMEM;
     qamw_codebook* cb = new (std::nothrow) qamw_codebook();
     if (!cb) return QAMW_ERR_NOMEM;
     cb->K = K;
-    cb->grid = t.grid;
+    cb->map = t.map;
     cb->n_candidates = t.n_candidates;
     cb->max_list = t.max_list;
     cb->n_overflow_cells = t.n_overflow_cells;
     cb->h_codebook.assign(codebook_host, codebook_host + 2 * K);
     cb->off_cells = size_t(K) * 8;
     cb->off_overflow = cb->off_cells + t.cells.size() * 2;
-    cb->off_lut = cb->off_overflow + t.overflow.size() * 2;
-    cb->blob_bytes = cb->off_lut + t.lut.size();
+    cb->blob_bytes = cb->off_overflow + t.overflow.size() * 2;
     std::vector<unsigned char> blob(cb->blob_bytes, 0);
     std::memcpy(blob.data(), codebook_host, size_t(K) * 8);
     std::memcpy(blob.data() + cb->off_cells, t.cells.data(), t.cells.size() * 2);
     if (!t.overflow.empty()) std::memcpy(blob.data() + cb->off_overflow, t.overflow.data(), t.overflow.size() * 2);
-    std::memcpy(blob.data() + cb->off_lut, t.lut.data(), t.lut.size());
     cudaError_t e = cudaGetDevice(&cb->device);
     if (e == cudaSuccess) e = cudaMalloc(&cb->d_blob, cb->blob_bytes);
     if (e == cudaSuccess) e = cudaMemcpy(cb->d_blob, blob.data(), cb->blob_bytes, cudaMemcpyHostToDevice);
@@ -1482,11 +1494,11 @@ extern "C" void qamw_codebook_destroy(qamw_codebook* cb) {
 
 extern "C" int qamw_codebook_table_info(const qamw_codebook* cb, int32_t* info_out) {
     if (!cb || !info_out) return QAMW_ERR_ARG;
-    info_out[0] = cb->grid;
+    info_out[0] = cb->map.grid;
     info_out[1] = cb->n_candidates;
     info_out[2] = cb->max_list;
     info_out[3] = cb->n_overflow_cells;
-    info_out[4] = int32_t((cb->off_lut - cb->off_overflow) / 2);
+    info_out[4] = int32_t((cb->blob_bytes - cb->off_overflow) / 2);
     info_out[5] = int32_t(cb->blob_bytes - size_t(cb->K) * 8);
     return QAMW_OK;
 }
@@ -1513,10 +1525,14 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     a.table = reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(cb->d_blob) + cb->off_cells);
     a.table_bytes = int(cb->blob_bytes - cb->off_cells);
     a.off_overflow = int(cb->off_overflow - cb->off_cells);
-    a.off_lut = int(cb->off_lut - cb->off_cells);
     a.K = p->K;
     a.log2K = ilog2(p->K);
-    a.grid = cb->grid;
+    a.grid = cb->map.grid;
+    a.map_zmax = cb->map.zmax;
+    a.map_c0 = cb->map.c0;
+    a.map_c1 = cb->map.c1;
+    a.map_c2 = cb->map.c2;
+    a.map_bias = 12582912.0f + float(cb->map.half);
     a.brute = (p->flags & QAMW_FLAG_BRUTE_FORCE) ? 1 : 0;
     a.packed = packed_out;
     a.packed_row_stride = p->packed_row_stride;

@@ -7,21 +7,20 @@
 // nearest-neighbour (Voronoi) region meets the cell, hence scanning the list
 // gives the same answer as scanning the codebook.
 //
-// Geometry.  Each axis is cut into 4096 fine bins of width 1/256 over [-8, 8)
-// (powers of two, so the device's fma(z, 256, 2048) is exact up to its final
-// rounding); the first and last bin also take everything beyond (the device
-// clamps the bin index), out to |z| < 16384.  A byte look-up table maps a fine
-// bin to one of `grid` coarse columns.  Column boundaries sit on fine-bin
-// edges: the inner ones near the quantiles of N(0, 2) -- the marginal of the
-// high-rate optimal point density f^(1/2) of a unit circular Gaussian source,
-// so that every inner cell holds about the same number of codewords -- followed
-// by a few geometrically widening tail columns for heavy-tailed inputs.
+// Geometry.  Both axes use the same map from a coordinate to a column, an odd
+// polynomial followed by rounding to the nearest integer (CellMap in
+// qamw_internal.h).  Its slope a (1 - z^2 / T)^2 follows the high-rate optimal
+// point density f^(1/2) of a unit circular Gaussian source closely enough that
+// the inner cells hold about the same number of codewords each, while the
+// device pays three fused multiply-adds per axis instead of a table look-up.
+// The coordinate is clamped to +-zmax first, so the outermost columns also take
+// everything beyond, out to |z| < 16384.
 //
 // Construction.  The Voronoi polygon of every codeword (clipped to the square
 // |z| <= 16384 and relaxed by a small slack, so it can only grow) is obtained by
 // clipping that square with the bisector half-planes of all other codewords.
 // A codeword is listed in a cell iff its polygon meets the cell's rectangle
-// enlarged by a margin that covers the rounding of the device's bin computation.
+// enlarged by a margin that covers the rounding of the device's f32 evaluation.
 #include <algorithm>
 #include <cmath>
 #include <cstring>
@@ -52,17 +51,6 @@ void clip_halfplane(const std::vector<Pt>& in, double a, double b, double c, std
             out->push_back(Pt{p.x + t * (q.x - p.x), p.y + t * (q.y - p.y)});
         }
     }
-}
-
-// Quantile of N(0, 2) by bisection on its CDF (1 + erf(x/2))/2; only used to place cell
-// boundaries, so its accuracy does not affect exactness.
-double quantile_n02(double p) {
-    double lo = -16.0, hi = 16.0;
-    for (int it = 0; it < 80; ++it) {
-        double mid = 0.5 * (lo + hi);
-        if (0.5 * (1.0 + std::erf(0.5 * mid)) < p) lo = mid; else hi = mid;
-    }
-    return 0.5 * (lo + hi);
 }
 
 // Voronoi polygon of codeword i inside [-kFar, kFar]^2, bisectors relaxed outwards by a slack.
@@ -97,66 +85,78 @@ void voronoi_polygon(const double* cb, int K, int i, std::vector<Pt>* poly, std:
 }  // namespace
 
 int default_grid(int K) {
-    int g = int(std::ceil(2.1 * std::sqrt(double(K)) / 8.0)) * 8;
-    return std::max(4, std::min(g, 192));
+    const int half = std::max(1, std::min(int(std::lround(1.08 * std::sqrt(double(K)))), 127));
+    return 2 * half + 1;
 }
 
-// Coarse boundaries in fine-bin units: edge[0] = 0 < ... < edge[grid] = kFineBins.
-static std::vector<int> make_edges(int grid) {
-    // number of widening tail columns per side (none for tiny grids)
-    const int tails = grid >= 24 ? 3 : (grid >= 12 ? 1 : 0);
-    const int core = grid - 2 * tails;
-    std::vector<double> pos;  // boundaries for z > 0, in z units
-    std::vector<double> inner;
-    for (int i = 1; i < core; ++i) inner.push_back(quantile_n02(double(i) / double(core)));
-    std::vector<double> all(inner);
-    if (tails > 0 && core >= 2) {
-        double last = inner.back();
-        double w = core >= 3 ? (inner[inner.size() - 1] - inner[inner.size() - 2]) * 1.5 : 1.0;
-        std::vector<double> up;
-        double e = last;
-        for (int t = 0; t < tails; ++t) {
-            e += w;
-            w *= 1.5;
-            up.push_back(std::min(e, 7.9 - 0.1 * (tails - 1 - t)));
-        }
-        for (double u : up) all.push_back(u);
-        for (double u : up) all.push_back(-u);
-    }
-    std::sort(all.begin(), all.end());
-    std::vector<int> edge(static_cast<size_t>(grid + 1), 0);
-    edge[0] = 0;
-    edge[size_t(grid)] = kFineBins;
-    for (int i = 1; i < grid; ++i) {
-        double q = (size_t(i - 1) < all.size()) ? all[size_t(i - 1)] : 7.9;
-        int e = int(std::lround(q * kFineScale + kFineOffset));
-        e = std::max(e, edge[size_t(i - 1)] + 1);
-        e = std::min(e, kFineBins - (grid - i));
-        edge[size_t(i)] = e;
-    }
-    return edge;
+// Slope a (1 - t / T)^2, t = z^2: value a z (1 - 2 t / (3 T) + t^2 / (5 T^2)), which reaches
+// (8 / 15) a sqrt(T) at z = sqrt(T).  `a` puts that maximum at half + 0.4, so the rounded value
+// stays within +-half; zmax stops a little before sqrt(T), where the slope is still safely positive
+// after the coefficients have been rounded to f32.
+constexpr double kMapT = 20.0;
+
+CellMap make_cell_map(int grid) {
+    CellMap m;
+    m.grid = grid;
+    m.half = (grid - 1) / 2;
+    const double root = std::sqrt(kMapT);
+    const double a = (double(m.half) + 0.4) / (root * 8.0 / 15.0);
+    m.c0 = float(a);
+    m.c1 = float(-2.0 * a / (3.0 * kMapT));
+    m.c2 = float(a / (5.0 * kMapT * kMapT));
+    m.zmax = float(0.98 * root);
+    return m;
 }
+
+double cell_map_value(const CellMap& m, double z) {
+    const double c = std::min(std::max(z, -double(m.zmax)), double(m.zmax));
+    const double t = c * c;
+    return c * (double(m.c0) + t * (double(m.c1) + t * double(m.c2)));
+}
+
+namespace {
+// Smallest z in [-zmax, zmax] with cell_map_value(z) >= v (the map is increasing there).
+double cell_map_inverse(const CellMap& m, double v) {
+    double lo = -double(m.zmax), hi = double(m.zmax);
+    if (cell_map_value(m, lo) >= v) return lo;
+    if (cell_map_value(m, hi) < v) return hi;
+    for (int it = 0; it < 100; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (cell_map_value(m, mid) < v) lo = mid; else hi = mid;
+    }
+    return hi;
+}
+}  // namespace
 
 bool build_cell_lists(const double* cb, int K, int grid, CellLists* out) {
-    if (grid < 1 || grid > 255) return false;
-    out->grid = grid;
-    std::vector<int> edge = make_edges(grid);
-    out->edges.resize(size_t(grid + 1));
-    for (int i = 0; i <= grid; ++i) out->edges[size_t(i)] = (double(edge[size_t(i)]) - kFineOffset) / kFineScale;
-    // the outermost columns also own everything beyond the fine range (the device clamps the bin)
-    out->edges[0] = -kFar;
-    out->edges[size_t(grid)] = kFar;
-    out->lut.assign(size_t(kFineBins), 0);
-    for (int i = 0; i < grid; ++i)
-        for (int f = edge[size_t(i)]; f < edge[size_t(i + 1)]; ++f) out->lut[size_t(f)] = uint8_t(i);
-    // 2^-10 of a fine bin covers the rounding of fma(z, 256, 2048) (at most 2^-12 of a bin)
-    const double margin = 1.0 / (1024.0 * kFineScale);
+    if (grid < 1 || grid > 255 || grid % 2 == 0) return false;
+    const CellMap m = make_cell_map(grid);
+    out->map = m;
+    {   // the map must be increasing on [-zmax, zmax] and stay inside +-(half + 0.45)
+        double prev = cell_map_value(m, 0.0);
+        for (int i = 1; i <= 4096; ++i) {
+            const double v = cell_map_value(m, double(m.zmax) * i / 4096.0);
+            if (!(v > prev)) return false;
+            prev = v;
+        }
+        if (!(prev < double(m.half) + 0.45)) return false;
+    }
+    // The device's f32 evaluation differs from the exact map by a few units of 2^-24 * half; a margin
+    // of 2^-8 of a column, on both sides of every boundary, covers it (and the tie rule of the
+    // rounding) many times over.
+    const double du = 1.0 / 256.0;
+    out->lo.assign(size_t(grid), 0.0);
+    out->hi.assign(size_t(grid), 0.0);
+    for (int j = 0; j < grid; ++j) {
+        const double v = double(j - m.half);
+        out->lo[size_t(j)] = j == 0 ? -kFar : cell_map_inverse(m, v - 0.5 - du);
+        out->hi[size_t(j)] = j == grid - 1 ? kFar : cell_map_inverse(m, v + 0.5 + du);
+    }
     out->lists.assign(size_t(grid) * grid, {});
     std::vector<Pt> poly, tmp, a, b;
-    auto column_of = [&](double z) {  // coarse column containing z (clamped like the device)
-        double f = std::floor(z * kFineScale + kFineOffset);
-        int fi = int(std::min(double(kFineBins - 1), std::max(0.0, f)));
-        return int(out->lut[size_t(fi)]);
+    auto column_of = [&](double z) {  // exact map; callers widen the range by one column
+        const int c = m.half + int(std::lround(cell_map_value(m, z)));
+        return std::min(grid - 1, std::max(0, c));
     };
     for (int i = 0; i < K; ++i) {
         voronoi_polygon(cb, K, i, &poly, &tmp);
@@ -166,12 +166,12 @@ bool build_cell_lists(const double* cb, int K, int grid, CellLists* out) {
             bx0 = std::min(bx0, p.x); bx1 = std::max(bx1, p.x);
             by0 = std::min(by0, p.y); by1 = std::max(by1, p.y);
         }
-        const int ix0 = column_of(bx0 - 2 * margin), ix1 = column_of(bx1 + 2 * margin);
-        const int iy0 = column_of(by0 - 2 * margin), iy1 = column_of(by1 + 2 * margin);
+        const int ix0 = std::max(0, column_of(bx0) - 1), ix1 = std::min(grid - 1, column_of(bx1) + 1);
+        const int iy0 = std::max(0, column_of(by0) - 1), iy1 = std::min(grid - 1, column_of(by1) + 1);
         for (int iy = iy0; iy <= iy1; ++iy)
             for (int ix = ix0; ix <= ix1; ++ix) {
-                const double x0 = out->edges[size_t(ix)] - margin, x1 = out->edges[size_t(ix + 1)] + margin;
-                const double y0 = out->edges[size_t(iy)] - margin, y1 = out->edges[size_t(iy + 1)] + margin;
+                const double x0 = out->lo[size_t(ix)], x1 = out->hi[size_t(ix)];
+                const double y0 = out->lo[size_t(iy)], y1 = out->hi[size_t(iy)];
                 clip_halfplane(poly, -1, 0, -x0, &a);          // x >= x0
                 if (a.empty()) continue;
                 clip_halfplane(a, 1, 0, x1, &b);               // x <= x1
@@ -197,9 +197,8 @@ bool build_cell_lists(const double* cb, int K, int grid, CellLists* out) {
 // ascending order (the last one repeated as padding).  A cell with more candidates
 // stores {0xFFFF, offset, count, 0} and its list goes to the overflow array.
 bool pack_search_table(const CellLists& cl, SearchTable* out) {
-    out->grid = cl.grid;
-    out->lut = cl.lut;
-    out->cells.assign(size_t(cl.grid) * cl.grid * 4, 0);
+    out->map = cl.map;
+    out->cells.assign(size_t(cl.map.grid) * cl.map.grid * 4, 0);
     out->overflow.clear();
     out->n_overflow_cells = 0;
     out->max_list = cl.max_list;
@@ -220,7 +219,8 @@ bool pack_search_table(const CellLists& cl, SearchTable* out) {
             ++out->n_overflow_cells;
         }
     }
-    while (out->overflow.size() % 8) out->overflow.push_back(0);  // keeps the next array 16-byte aligned
+    // the device copies the table in 16-byte pieces: pad it to a whole number of them
+    while ((out->cells.size() + out->overflow.size()) % 8) out->overflow.push_back(0);
     return true;
 }
 
@@ -228,8 +228,8 @@ bool choose_search_table(const float* codebook, int K, int grid, size_t budget_b
     std::vector<double> cb(static_cast<size_t>(2 * K), 0.0);
     for (int i = 0; i < 2 * K; ++i) cb[size_t(i)] = double(codebook[i]);
     int g = grid > 0 ? grid : default_grid(K);
-    for (; g >= 1; g = (grid > 0 || g <= 8) ? g - 1 : g - 8) {
-        if (size_t(g) * g * 8 + kFineBins > budget_bytes) {
+    for (; g >= 1; g -= 2) {
+        if (size_t(g) * g * 8 > budget_bytes) {
             if (grid > 0) return false;
             continue;
         }
@@ -249,19 +249,25 @@ bool choose_search_table(const float* codebook, int K, int grid, size_t budget_b
 using namespace qamw;
 
 extern "C" int qamw_search_table_build(const float* codebook_host, int K, int grid, size_t budget_bytes,
-                                       uint8_t* lut_out, uint16_t* cells_out, size_t cells_cap,
+                                       float* map_out, uint16_t* cells_out, size_t cells_cap,
                                        uint16_t* overflow_out, size_t overflow_cap, int32_t* info_out) {
     if (!codebook_host || !info_out) return QAMW_ERR_ARG;
     if (K < 1 || K > QAMW_MAX_K || !is_pow2(K)) return QAMW_ERR_SHAPE;
+    if (grid < 0 || grid > 255 || (grid > 0 && grid % 2 == 0)) return QAMW_ERR_ARG;
     SearchTable t;
     if (!choose_search_table(codebook_host, K, grid, budget_bytes, &t)) return QAMW_ERR_NOMEM;
-    info_out[0] = t.grid;
+    info_out[0] = t.map.grid;
     info_out[1] = t.n_candidates;
     info_out[2] = t.max_list;
     info_out[3] = t.n_overflow_cells;
     info_out[4] = int32_t(t.overflow.size());
     info_out[5] = int32_t(t.bytes());
-    if (lut_out) std::memcpy(lut_out, t.lut.data(), t.lut.size());
+    if (map_out) {
+        map_out[0] = t.map.zmax;
+        map_out[1] = t.map.c0;
+        map_out[2] = t.map.c1;
+        map_out[3] = t.map.c2;
+    }
     if (cells_out) {
         if (cells_cap < t.cells.size()) return QAMW_ERR_NOMEM;
         std::memcpy(cells_out, t.cells.data(), t.cells.size() * 2);

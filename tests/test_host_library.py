@@ -68,11 +68,22 @@ def test_library_trainer_is_a_lloyd_fixed_point_like_the_oracles(orc, K):
     assert np.all(np.diff(r2) >= 0)  # sorted by radius
 
 
-def _table_search(cb, lut, cells, ovf, grid, z):
-    """What the device's table search computes, in numpy (f32 bin arithmetic, f64 distances)."""
-    f = (z.astype(np.float32) * np.float32(256.0) + np.float32(2048.0)).astype(np.float32)
-    b = np.clip(np.floor(f), 0, 4095).astype(np.int64)
-    rec = cells[lut[b[:, 1]].astype(np.int64) * grid + lut[b[:, 0]].astype(np.int64)]
+def _columns(cmap, grid, z, nudge=0.0):
+    """The cell map of include/qamw.h in f32 steps (numpy has no fused multiply-add: a product and a sum
+    rounded separately land, at worst, in the neighbouring column, whose list holds the answer too).
+    `nudge` moves the value by a fraction of a column before the rounding."""
+    zmax, c0, c1, c2 = (np.float32(v) for v in cmap)
+    c = np.minimum(np.maximum(z.astype(np.float32), -zmax), zmax)
+    t = c * c
+    u = c * (c0 + t * (c1 + t * c2))
+    col = np.rint(u.astype(np.float64) + nudge).astype(np.int64) + (grid - 1) // 2
+    return np.clip(col, 0, grid - 1)
+
+
+def _table_search(cb, cmap, cells, ovf, grid, z, nudge=0.0):
+    """What the device's table search computes, in numpy (f32 cell arithmetic, f64 distances)."""
+    col = _columns(cmap, grid, z, nudge)
+    rec = cells[col[:, 1] * grid + col[:, 0]]
     out = np.empty(len(z), np.int64)
     for i in range(len(z)):
         r = rec[i]
@@ -83,36 +94,55 @@ def _table_search(cb, lut, cells, ovf, grid, z):
     return out
 
 
-@pytest.mark.parametrize("K,grid", [(64, 0), (256, 0), (2048, 0), (2048, 40), (4096, 0)])
+@pytest.mark.parametrize("K,grid", [(64, 0), (256, 0), (2048, 0), (2048, 41), (4096, 0)])
 def test_search_table_is_exact(K, grid):
     """Every cell lists all codewords whose nearest-neighbour region meets it: scanning the list
     gives the exhaustive answer, for Gaussian points, heavy tails and points far outside."""
     cb = load_golden_codebook(K)
-    lut, cells, ovf, info = q.search_table_build(cb, grid, 1 << 20)
+    cmap, cells, ovf, info = q.search_table_build(cb, grid, 1 << 20)
     g = int(info[0])
-    assert cells.shape == (g * g, 4) and int(info[5]) == 4096 + cells.size * 2 + (0 if info[4] == 0 else ovf.size * 2)
+    assert g % 2 == 1 and cells.shape == (g * g, 4) and int(info[5]) == cells.size * 2 + int(info[4]) * 2
+    assert int(info[5]) % 16 == 0  # the device copies it in 16-byte pieces
     rng = np.random.default_rng(K + grid)
     z = np.concatenate([rng.standard_normal((6000, 2)), 3 * rng.standard_t(3, (3000, 2)),
                         rng.uniform(-9, 9, (2000, 2)), 1000 * rng.standard_normal((500, 2)),
                         cb[:64].astype(np.float64) + 1e-4 * rng.standard_normal((64, 2))]).astype(np.float32)
     z = z[np.abs(z).max(1) < 16000]
-    got = _table_search(cb, lut, cells, ovf, g, z)
     d = ((z[:, None, :].astype(np.float64) - cb[None].astype(np.float64)) ** 2).sum(2)
     best = d.argmin(1)
     part = np.partition(d, 1, axis=1)
     near_tie = (part[:, 1] - part[:, 0]) < 1e-6 * part[:, 1]
-    assert np.all((got == best) | near_tie)
+    # the lists also cover a point that rounding carries into the neighbouring column or row
+    for nudge in (0.0, 1 / 512, -1 / 512):
+        got = _table_search(cb, cmap, cells, ovf, g, z, nudge)
+        assert np.all((got == best) | near_tie)
 
 
 def test_default_table_fits_the_encoder_and_explicit_grid_is_honoured():
     cb = load_golden_codebook(2048)
     _, _, _, info = q.search_table_build(cb, 0, 77 * 1024)
     assert info[5] <= 77 * 1024 and info[2] >= 4  # longest list beyond 4: overflow lists exist
-    _, cells, _, info = q.search_table_build(cb, 24, 1 << 20)
-    assert info[0] == 24 and cells.shape[0] == 576
+    _, cells, _, info = q.search_table_build(cb, 25, 1 << 20)
+    assert info[0] == 25 and cells.shape[0] == 625
     with pytest.raises(q.QamwError) as e:
-        q.search_table_build(cb, 200, 64 * 1024)
+        q.search_table_build(cb, 201, 64 * 1024)
     assert e.value.code == q.ERR_NOMEM
+    with pytest.raises(q.QamwError) as e:
+        q.search_table_build(cb, 24, 1 << 20)  # the grid side is odd
+    assert e.value.code == q.ERR_ARG
+
+
+def test_cell_map_is_increasing_and_stays_inside_the_grid():
+    cb = load_golden_codebook(256)
+    for grid in (3, 25, 99, 255):
+        cmap, _, _, info = q.search_table_build(cb, grid, 1 << 22)
+        z = np.linspace(-float(cmap[0]) * 1.5, float(cmap[0]) * 1.5, 20001).astype(np.float32)
+        zz = np.stack([z, z], 1)
+        col = _columns(cmap, grid, zz)[:, 0]
+        assert np.all(np.diff(col) >= 0) and col.min() == 0 and col.max() == grid - 1
+        assert np.all(np.diff(col) <= 1)  # no column is skipped at this sampling density
+        far = np.array([[-1e30, 1e30], [np.inf, -np.inf]], np.float32)
+        assert _columns(cmap, grid, far).tolist() == [[0, grid - 1], [grid - 1, 0]]
 
 
 def test_argument_errors_are_reported_before_any_launch():
