@@ -516,7 +516,7 @@ __device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
 
 struct SearchSmem {       // all fields are shared-memory byte addresses
     uint32_t cb;          // codebook copies, already offset to this lane's copy
-    int cb_shift;         // log2 of the byte distance between consecutive entries (3 + log2c)
+    uint32_t cb_stride;   // byte distance between consecutive entries (8 << log2c)
     uint32_t cells;       // grid*grid records of 8 bytes; minus 8 * (grid + 1) * kMagicBits, see search_cell
     uint32_t overflow;    // u16 lists
     uint32_t grid;
@@ -529,7 +529,7 @@ struct SearchSmem {       // all fields are shared-memory byte addresses
 constexpr uint32_t kMagicBits = 0x4B400000u;  // bit pattern of 1.5 * 2^23 = 12582912.0f
 
 __device__ __forceinline__ float2 codeword(const SearchSmem& s, int k) {
-    return lds_f32x2(s.cb + (uint32_t(k) << s.cb_shift));
+    return lds_f32x2(s.cb + uint32_t(k) * s.cb_stride);
 }
 
 // Squared distance in direct form, one rounding per operation: f32(f32(dx^2) + f32(dy^2)); the two
@@ -588,13 +588,11 @@ __device__ __forceinline__ int search_cell(const SearchSmem& s, float zx, float 
     // The list is ascending and padded by repeating its last entry (a repeated slot cannot win).
     const float2 c0 = codeword(s, k0), c1 = codeword(s, k1), c2 = codeword(s, k2), c3 = codeword(s, k3);
     const float d0 = dist2(c0, zx, zy), d1 = dist2(c1, zx, zy), d2 = dist2(c2, zx, zy), d3 = dist2(c3, zx, zy);
-    // lowest slot (= lowest index) among equal distances
-    float best = d0;
-    int arg = k0;
-    if (d1 < best) { best = d1; arg = k1; }
-    if (d2 < best) { best = d2; arg = k2; }
-    if (d3 < best) { best = d3; arg = k3; }
-    return arg;
+    // lowest slot (= lowest index) among equal distances: a later slot wins only when strictly closer
+    const bool s1 = d1 < d0, s3 = d3 < d2;
+    const float da = s1 ? d1 : d0, db = s3 ? d3 : d2;
+    const int ka = s1 ? k1 : k0, kb = s3 ? k3 : k2;
+    return db < da ? kb : ka;
 }
 
 __device__ __noinline__ int search_table(const SearchSmem& s, float zx, float zy) {
@@ -709,7 +707,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
 
     SearchSmem s;
     s.cb = smem_addr(smem) + 8u * (threadIdx.x & ((1 << a.log2c) - 1));
-    s.cb_shift = 3 + a.log2c;
+    s.cb_stride = 8u << a.log2c;
     s.cells = smem_addr(table) - 8u * kMagicBits * uint32_t(a.grid + 1);
     s.overflow = smem_addr(table + a.off_overflow);
     s.grid = uint32_t(a.grid);
@@ -800,16 +798,18 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
             for (int rr = 0; rr < 4; ++rr) {
                 const int k0 = 4 * Layout<LOG2B_T>::octet_after(tid_g, rr);
                 if (k0 >= n_pairs) continue;
-                unsigned long long packed4 = 0ull;
+                uint32_t v[4];
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
                     const float2 z = zst[(rr * 4 + p) * 32];
-                    int v;
-                    if (MODE == 2) v = search_exhaustive(s, z.x, z.y);
-                    else if (MODE == 1) v = search_table(s, z.x, z.y);
-                    else v = search_cell(s, z.x, z.y);
-                    if (k0 + p < n_pairs) packed4 |= (unsigned long long)uint32_t(v) << (p * B);
+                    if (MODE == 2) v[p] = uint32_t(search_exhaustive(s, z.x, z.y));
+                    else if (MODE == 1) v[p] = uint32_t(search_table(s, z.x, z.y));
+                    else v[p] = uint32_t(search_cell(s, z.x, z.y));
                 }
+                // two indices fit a 32-bit word (B <= 12)
+                unsigned long long packed4 =
+                    (unsigned long long)(v[0] | (v[1] << B)) | ((unsigned long long)(v[2] | (v[3] << B)) << (2 * B));
+                if (k0 + 4 > n_pairs) packed4 &= (1ull << ((n_pairs - k0) * B)) - 1ull;  // the row ends inside this octet
                 oct_s[stage_slot((k0 >> 2) - oct0)] = packed4;
             }
             __syncwarp();
