@@ -19,15 +19,19 @@ inline int ilog2(int64_t v) {
 // Column (and, with the same map, row) of the search grid that holds coordinate z:
 //     c = min(max(z, -zmax), zmax);  t = c * c;
 //     column = half + rn(c * (c0 + t * (c1 + t * c2)))            (rn: to nearest integer)
-// an odd polynomial whose slope falls like (1 - t / T)^2: cells are narrow where a Gaussian source
-// puts its codewords and widen towards zmax; the outermost columns take everything beyond.  The
+// an odd polynomial with slope a ((1 - t / T)^2 + eps): cells are narrow where a Gaussian source
+// puts its codewords, widen up to sqrt(T) and get a few more columns between there and
+// zmax = rho sqrt(T) for heavy-tailed inputs; the outermost columns take everything beyond.  The
 // device evaluates it in f32 (three fused multiply-adds, the last one onto 1.5 * 2^23 + half, which
 // leaves the integer in the low mantissa bits).  grid = 2 * half + 1 is odd.
 struct CellMap {
     int grid = 0, half = 0;
     float zmax = 0.f, c0 = 0.f, c1 = 0.f, c2 = 0.f;
 };
-CellMap make_cell_map(int grid);
+struct MapShape {
+    double T = 18.0, eps = 0.02, rho = 1.25;
+};
+CellMap make_cell_map(int grid, const MapShape& shape);
 // The map in exact arithmetic on the f32 coefficients (before rounding to an integer).
 double cell_map_value(const CellMap& m, double z);
 
@@ -53,8 +57,18 @@ struct SearchTable {
     size_t bytes() const { return cells.size() * 2 + overflow.size() * 2; }
 };
 
+// Nearest-neighbour (Voronoi) polygons of all codewords, clipped to |z| <= 16384: the vertices of
+// codeword i are xy[2 * start[i]] .. xy[2 * start[i + 1]).
+struct VoronoiSet {
+    std::vector<int> start;
+    std::vector<double> xy;
+};
+void voronoi_polygons(const double* cb, int K, VoronoiSet* out);
+
 int default_grid(int K);
-bool build_cell_lists(const double* cb, int K, int grid, CellLists* out);
+bool build_cell_lists(const VoronoiSet& vs, int K, const CellMap& map, CellLists* out);
+bool build_cell_lists(const double* cb, int K, int grid, CellLists* out);  // default map shape
+double overflow_cost(const CellLists& cl);
 bool pack_search_table(const CellLists& cl, SearchTable* out);
 
 // grid > 0 (odd): exactly that grid (fails if it does not fit); grid == 0: the default grid for K,

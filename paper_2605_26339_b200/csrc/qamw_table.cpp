@@ -89,22 +89,21 @@ int default_grid(int K) {
     return 2 * half + 1;
 }
 
-// Slope a (1 - t / T)^2, t = z^2: value a z (1 - 2 t / (3 T) + t^2 / (5 T^2)), which reaches
-// (8 / 15) a sqrt(T) at z = sqrt(T).  `a` puts that maximum at half + 0.4, so the rounded value
-// stays within +-half; zmax stops a little before sqrt(T), where the slope is still safely positive
-// after the coefficients have been rounded to f32.
-constexpr double kMapT = 20.0;
-
-CellMap make_cell_map(int grid) {
+// Slope a ((1 - t / T)^2 + eps), t = z^2: the value a z (1 + eps - 2 t / (3 T) + t^2 / (5 T^2)) is
+// increasing everywhere.  Up to sqrt(T) the cells widen like the spacing of the codewords of a
+// Gaussian source; between sqrt(T) and zmax = rho sqrt(T) the slope rises again, which spends a few
+// columns on the far tail, where heavy-tailed inputs (outlier channels) put many of their pairs.
+// `a` makes the value at zmax half + 0.4, so the rounded value stays within +-half.
+CellMap make_cell_map(int grid, const MapShape& shape) {
     CellMap m;
     m.grid = grid;
     m.half = (grid - 1) / 2;
-    const double root = std::sqrt(kMapT);
-    const double a = (double(m.half) + 0.4) / (root * 8.0 / 15.0);
-    m.c0 = float(a);
-    m.c1 = float(-2.0 * a / (3.0 * kMapT));
-    m.c2 = float(a / (5.0 * kMapT * kMapT));
-    m.zmax = float(0.98 * root);
+    const double T = shape.T, zmax = shape.rho * std::sqrt(T), t = zmax * zmax;
+    const double a = (double(m.half) + 0.4) / (zmax * (1.0 + shape.eps - 2.0 * t / (3.0 * T) + t * t / (5.0 * T * T)));
+    m.c0 = float(a * (1.0 + shape.eps));
+    m.c1 = float(-2.0 * a / (3.0 * T));
+    m.c2 = float(a / (5.0 * T * T));
+    m.zmax = float(zmax);
     return m;
 }
 
@@ -126,11 +125,27 @@ double cell_map_inverse(const CellMap& m, double v) {
     }
     return hi;
 }
+
+double normal_cdf(double x, double sd) { return 0.5 * std::erfc(-x / (sd * std::sqrt(2.0))); }
 }  // namespace
 
-bool build_cell_lists(const double* cb, int K, int grid, CellLists* out) {
+void voronoi_polygons(const double* cb, int K, VoronoiSet* out) {
+    out->start.assign(size_t(K) + 1, 0);
+    out->xy.clear();
+    std::vector<Pt> poly, tmp;
+    for (int i = 0; i < K; ++i) {
+        voronoi_polygon(cb, K, i, &poly, &tmp);
+        for (const Pt& p : poly) {
+            out->xy.push_back(p.x);
+            out->xy.push_back(p.y);
+        }
+        out->start[size_t(i) + 1] = int(out->xy.size() / 2);
+    }
+}
+
+bool build_cell_lists(const VoronoiSet& vs, int K, const CellMap& m, CellLists* out) {
+    const int grid = m.grid;
     if (grid < 1 || grid > 255 || grid % 2 == 0) return false;
-    const CellMap m = make_cell_map(grid);
     out->map = m;
     {   // the map must be increasing on [-zmax, zmax] and stay inside +-(half + 0.45)
         double prev = cell_map_value(m, 0.0);
@@ -153,13 +168,15 @@ bool build_cell_lists(const double* cb, int K, int grid, CellLists* out) {
         out->hi[size_t(j)] = j == grid - 1 ? kFar : cell_map_inverse(m, v + 0.5 + du);
     }
     out->lists.assign(size_t(grid) * grid, {});
-    std::vector<Pt> poly, tmp, a, b;
+    std::vector<Pt> poly, a, b;
     auto column_of = [&](double z) {  // exact map; callers widen the range by one column
         const int c = m.half + int(std::lround(cell_map_value(m, z)));
         return std::min(grid - 1, std::max(0, c));
     };
     for (int i = 0; i < K; ++i) {
-        voronoi_polygon(cb, K, i, &poly, &tmp);
+        poly.clear();
+        for (int v = vs.start[size_t(i)]; v < vs.start[size_t(i) + 1]; ++v)
+            poly.push_back(Pt{vs.xy[2 * size_t(v)], vs.xy[2 * size_t(v) + 1]});
         if (poly.empty()) continue;
         double bx0 = INFINITY, bx1 = -INFINITY, by0 = INFINITY, by1 = -INFINITY;
         for (const Pt& p : poly) {
@@ -191,6 +208,35 @@ bool build_cell_lists(const double* cb, int K, int grid, CellLists* out) {
         out->n_candidates += int(l.size());
     }
     return true;
+}
+
+bool build_cell_lists(const double* cb, int K, int grid, CellLists* out) {
+    VoronoiSet vs;
+    voronoi_polygons(cb, K, &vs);
+    return build_cell_lists(vs, K, make_cell_map(grid, MapShape{}), out);
+}
+
+// Expected number of list entries that a point has to scan beyond the four of a cell record, for
+// points drawn from 0.9 N(0, I) + 0.1 N(0, 4 I): pairs after the rotation are close to Gaussian,
+// with a heavier tail where an outlier channel dominates its block.  Used to rank map shapes.
+double overflow_cost(const CellLists& cl) {
+    const int grid = cl.map.grid;
+    double cost = 0.0;
+    for (int comp = 0; comp < 2; ++comp) {
+        const double sd = comp ? 2.0 : 1.0, weight = comp ? 0.1 : 0.9;
+        std::vector<double> mass(static_cast<size_t>(grid), 0.0);
+        for (int j = 0; j < grid; ++j) {  // columns without their margins: split at the midpoints of the overlaps
+            const double lo = j == 0 ? -INFINITY : 0.5 * (cl.lo[size_t(j)] + cl.hi[size_t(j) - 1]);
+            const double hi = j == grid - 1 ? INFINITY : 0.5 * (cl.hi[size_t(j)] + cl.lo[size_t(j) + 1]);
+            mass[size_t(j)] = (std::isinf(hi) ? 1.0 : normal_cdf(hi, sd)) - (std::isinf(lo) ? 0.0 : normal_cdf(lo, sd));
+        }
+        for (int iy = 0; iy < grid; ++iy)
+            for (int ix = 0; ix < grid; ++ix) {
+                const size_t n = cl.lists[size_t(iy) * grid + ix].size();
+                if (n > 4) cost += weight * mass[size_t(ix)] * mass[size_t(iy)] * double(n);
+            }
+    }
+    return cost;
 }
 
 // Device layout: one 8-byte record per cell holding up to four candidate indices in
@@ -227,17 +273,32 @@ bool pack_search_table(const CellLists& cl, SearchTable* out) {
 bool choose_search_table(const float* codebook, int K, int grid, size_t budget_bytes, SearchTable* out) {
     std::vector<double> cb(static_cast<size_t>(2 * K), 0.0);
     for (int i = 0; i < 2 * K; ++i) cb[size_t(i)] = double(codebook[i]);
-    int g = grid > 0 ? grid : default_grid(K);
-    for (; g >= 1; g -= 2) {
-        if (size_t(g) * g * 8 > budget_bytes) {
-            if (grid > 0) return false;
-            continue;
-        }
-        CellLists cl;
-        SearchTable t;
-        if (build_cell_lists(cb.data(), K, g, &cl) && pack_search_table(cl, &t) && t.bytes() <= budget_bytes) {
-            *out = std::move(t);
-            return true;
+    VoronoiSet vs;
+    voronoi_polygons(cb.data(), K, &vs);
+    // A few map shapes around the default: how many cells end up with more than four candidates
+    // depends on how the column boundaries happen to fall between the codewords of this codebook.
+    std::vector<MapShape> shapes;
+    for (double T : {17.0, 18.0, 19.0})
+        for (double eps : {0.015, 0.02})
+            for (double rho : {1.22, 1.27}) shapes.push_back(MapShape{T, eps, rho});
+    for (int g = grid > 0 ? grid : default_grid(K); g >= 1; g -= 2) {
+        if (size_t(g) * g * 8 <= budget_bytes) {
+            bool found = false;
+            double best = INFINITY;
+            for (const MapShape& shape : shapes) {
+                CellLists cl;
+                SearchTable t;
+                if (!build_cell_lists(vs, K, make_cell_map(g, shape), &cl) || !pack_search_table(cl, &t) ||
+                    t.bytes() > budget_bytes)
+                    continue;
+                const double cost = overflow_cost(cl);
+                if (cost < best) {
+                    best = cost;
+                    *out = std::move(t);
+                    found = true;
+                }
+            }
+            if (found) return true;
         }
         if (grid > 0) return false;
     }
