@@ -85,7 +85,9 @@ void voronoi_polygon(const double* cb, int K, int i, std::vector<Pt>* poly, std:
 }  // namespace
 
 int default_grid(int K) {
-    const int half = std::max(1, std::min(int(std::lround(1.08 * std::sqrt(double(K)))), 127));
+    // about 2.2 sqrt(K) columns, and never fewer than 31: a small table is cheap, and with fewer
+    // columns the outermost ones are crowded enough to overflow
+    const int half = std::max(15, std::min(int(std::lround(1.08 * std::sqrt(double(K)))), 127));
     return 2 * half + 1;
 }
 
