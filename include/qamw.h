@@ -125,7 +125,8 @@ int qamw_status_to_error(int32_t status_word);
  * codewords and widening outwards; every cell lists all codewords whose nearest-neighbour region
  * can meet the cell, so a scan of the list returns what a scan of the whole codebook returns.
  * The outermost cells reach to |z| < 16384; points beyond are scanned exhaustively.  grid = 0
- * picks a default (about 2.2 sqrt(K)); an explicit grid must be odd and at most 255, else
+ * picks a default (about 2.2 sqrt(K), at least 31, shrunk until the table fits next to the encoder's
+ * other shared memory); an explicit grid must be odd and at most 255, else
  * QAMW_ERR_ARG.  Synchronous.
  * *out must be released with qamw_codebook_destroy on the same device. */
 int qamw_codebook_create(const float* codebook_host, int K, int grid, qamw_codebook** out);

@@ -284,6 +284,35 @@ def test_extreme_z_falls_back_to_exhaustive_search(orc):
     assert not np.any((idx_gpu != enc["idx"]) & ~exempt)
 
 
+@pytest.mark.parametrize("K,grid", [(256, 3), (256, 9), (256, 117), (2048, 41)])
+def test_explicit_search_grids(orc, K, grid):
+    """A coarse grid sends nearly every point through the overflow lists, a fine one through cells
+    with a single candidate; the indices are the oracle's either way, also for heavy-tailed pairs
+    that land in the outermost columns."""
+    W, act = _make(24, 1024, torch.float32, 300 + grid)
+    # a few huge entries per row: the pairs of their blocks spread far beyond the Gaussian range
+    W[torch.rand(W.shape, generator=torch.Generator().manual_seed(grid)) < 0.004] *= 40.0
+    cb_host = load_golden_codebook(K)
+    cb = q.Codebook(cb_host, grid=grid)
+    assert int(cb.table_info()[0]) == grid
+    if grid <= 9:
+        assert int(cb.table_info()[3]) > grid * grid // 2  # most cells overflow
+    signs = q.make_signs(q.DEFAULT_SIGN_SEED, 1024)
+    sigma, _ = orc.calibrate(W.numpy(), 128, None, signs)
+    p = q.make_params(W.to(DEV), 24, 1024, 128, K)
+    packed = torch.zeros((24, p.packed_row_stride), dtype=torch.uint8, device=DEV)
+    norm = torch.empty(24, dtype=torch.float32, device=DEV)
+    q.encode(W.to(DEV), p, None, torch.from_numpy(signs).to(DEV), torch.from_numpy(sigma).to(DEV), cb, packed, norm)
+    enc = orc.encode(W.numpy(), 128, cb_host, None, signs, sigma, packed_row_stride=p.packed_row_stride,
+                     diagnostics=True)
+    assert np.abs(enc["z"]).max() > 4.5  # beyond the polynomial part of the cell map
+    B = int(np.log2(K))
+    idx_gpu = np.stack([orc.unpack_row(r, 512, B) for r in packed.cpu().numpy()])
+    exempt = (enc["d2_second"] - enc["d2_best"]) < 1e-6 * enc["d2_second"]
+    assert not np.any((idx_gpu != enc["idx"]) & ~exempt)
+    assert np.array_equal(norm.cpu().numpy(), enc["row_norm"])
+
+
 @pytest.mark.parametrize("name,mid", [("cfg3", 0), ("cfg3", 4), ("cfg3", 6), ("cfg1", 6), ("cfg2", 1)])
 def test_full_size_matrices_sampled_rows(orc, name, mid):
     """Benchmark-size matrices in the benchmark's launch configuration (whole matrix on the device,
