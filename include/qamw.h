@@ -55,7 +55,7 @@ extern "C" {
 #define QAMW_DTYPE_BF16 1
 
 #define QAMW_FLAG_BRUTE_FORCE 1u /* encode: exhaustive search over all K instead of the cell table */
-#define QAMW_FLAG_HALF_DEVICE 2u /* encode, decode, rotate: use every second SM only, so that two calls issued on
+#define QAMW_FLAG_HALF_DEVICE 2u /* encode, decode, rotate, calibrate: half as many blocks, so that two calls issued on
                                     different streams run side by side and each one's start-up (tables and
                                     per-column constants into shared memory and registers) hides behind the other */
 
@@ -161,7 +161,8 @@ size_t qamw_calibrate_workspace_bytes(const qamw_params* p);
  * rows i = floor(t*d_out/n), rows of zero norm skipped, y as in the arithmetic contract above;
  * floored at 1e-4/sqrt(d_in); 1/sqrt(d_in) when no row qualifies.  The column means are
  * accumulated in double, per thread block and then in a fixed order, so the result is
- * reproducible.  workspace: device scratch of at least qamw_calibrate_workspace_bytes(p) bytes,
+ * reproducible (QAMW_FLAG_HALF_DEVICE groups the rows differently: the double sums, and rarely the
+ * last bit of a sigma, can differ between the two settings).  workspace: device scratch of at least qamw_calibrate_workspace_bytes(p) bytes,
  * 8-byte aligned, overwritten.  status_out: device int32, bit 0 set if a row norm was not finite
  * (may be NULL). */
 int qamw_calibrate(const void* W, const qamw_params* p, const float* chan_scale, const int8_t* signs,

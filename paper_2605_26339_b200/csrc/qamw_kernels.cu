@@ -1587,7 +1587,7 @@ struct CalibPlan {
 CalibPlan calib_plan(const qamw_params* p, const RowGeom& g) {
     CalibPlan c;
     c.n_rows = std::min(p->d_out, QAMW_CALIB_MAX_ROWS);
-    c.blocks = std::max(1, std::min(148, (c.n_rows + g.groups - 1) / g.groups));
+    c.blocks = std::max(1, std::min(std::min(148, grid_limit(p)), (c.n_rows + g.groups - 1) / g.groups));
     c.total_groups = c.blocks * g.groups;
     c.pair_stride = ((p->d_in / 2 + 3) / 4) * 4;
     c.bytes = (size_t(c.total_groups) * c.pair_stride + size_t(c.total_groups)) * sizeof(double);
