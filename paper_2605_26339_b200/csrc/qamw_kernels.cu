@@ -482,9 +482,12 @@ __device__ __forceinline__ void fill_codebook_copies(float2* dst, const float2* 
             if (log2c == 0) {
                 dst[i] = c[u];
             } else {
+                // 2^m 16-byte pieces per entry; consecutive lanes own consecutive entries, so a lane
+                // starts at the piece that puts the warp's stores on all banks at once
                 float4* d4 = reinterpret_cast<float4*>(dst + (size_t(i) << log2c));
                 const float4 v = make_float4(c[u].x, c[u].y, c[u].x, c[u].y);
-                for (int k = 0; k < (1 << (log2c - 1)); ++k) d4[k] = v;
+                const int m = log2c - 1, first = (threadIdx.x & 31) >> (3 - m);
+                for (int k = 0; k < (1 << m); ++k) d4[(first + k) & ((1 << m) - 1)] = v;
             }
         }
     }
