@@ -251,7 +251,7 @@ def test_no_channel_scaling_and_brute_force_flag(orc):
 def test_zero_outlier_and_nonfinite_rows(orc):
     W, act = _make(12, 512, torch.float32, 13, student=False)
     W[2] = 0
-    W[5, 17] = 3.0e4  # one huge entry: its block's points leave the table's [-8, 8) square
+    W[5, 17] = 3.0e4  # one huge entry: its block's points land in the outermost cells of the table
     c = Case(orc, W, act, 0.0, 128, 256)
     c.check_all()
     assert c.norm[2] == 0 and not orc.bf16_to_f32(c.what_full[2]).any()
@@ -267,18 +267,21 @@ def test_zero_outlier_and_nonfinite_rows(orc):
     assert not np.any((idx_gpu != c.enc["idx"][ok]) & ~exempt)
 
 
-def test_extreme_z_falls_back_to_exhaustive_search(orc):
-    """sigma far too small drives every point outside the table; the exhaustive fallback must agree."""
+@pytest.mark.parametrize("sigma0,z_min", [(1e-3, 8.0), (1e-5, 16000.0)])
+def test_extreme_z(orc, sigma0, z_min):
+    """sigma far too small: at 1e-3 the points land in the outermost cells of the table (|z| up to
+    some hundreds); at 1e-5 the reciprocal scale is large enough for the encoder to run its variant
+    with the reach check, and the points beyond |z| = 16000 go through the exhaustive scan."""
     W, act = _make(6, 256, torch.float32, 17, student=False)
     cb_host, cb = _codebook(orc, 256)
     signs = q.make_signs(q.DEFAULT_SIGN_SEED, 256)
-    sigma = np.full(128, 1e-3, np.float32)
+    sigma = np.full(128, sigma0, np.float32)
     p = q.make_params(W.to(DEV), 6, 256, 64, 256)
     packed = torch.zeros((6, p.packed_row_stride), dtype=torch.uint8, device=DEV)
     norm = torch.empty(6, dtype=torch.float32, device=DEV)
     q.encode(W.to(DEV), p, None, torch.from_numpy(signs).to(DEV), torch.from_numpy(sigma).to(DEV), cb, packed, norm)
     enc = orc.encode(W.numpy(), 64, cb_host, None, signs, sigma, packed_row_stride=p.packed_row_stride, diagnostics=True)
-    assert np.abs(enc["z"]).max() > 8
+    assert np.abs(enc["z"]).max() > z_min
     idx_gpu = np.stack([orc.unpack_row(r, 128, 8) for r in packed.cpu().numpy()])
     exempt = (enc["d2_second"] - enc["d2_best"]) < 1e-6 * enc["d2_second"]
     assert not np.any((idx_gpu != enc["idx"]) & ~exempt)
