@@ -1114,59 +1114,70 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
                                __fdiv_rn(sgn[r][2 * i + 1] * a.inv_sqrt_b, cs[r][2 * i + 1]));
     __syncthreads();
 
-    int buf = 0;
-    for (; row < g.d_out; row += row_step, buf ^= 1) {
-        const float rn = a.row_norm[row];
-        cp_async_wait_all();
-        __syncwarp();  // every lane's part of this row has landed; the other buffer is no longer read
-        if (row + row_step < g.d_out) issue_row(row + row_step, buf ^ 1);
-        const uint32_t* in = reinterpret_cast<const uint32_t*>(stage + buf * a.stage_bytes);
-        f32x2 P[4][4];
+    // The row loop exists twice.  When the rows allow 16-byte accesses (d_in a multiple of 8), octets
+    // beyond the end of the row are decoded like the others instead of being tested for: their pair
+    // scales are 0, so whatever index the staging buffer holds for them decodes to 0, they belong to
+    // Hadamard blocks that lie wholly beyond the row, and only their stores are suppressed.
+    auto rows = [&](auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
+        int buf = 0;
+        for (; row < g.d_out; row += row_step, buf ^= 1) {
+            const float rn = a.row_norm[row];
+            cp_async_wait_all();
+            __syncwarp();  // every lane's part of this row has landed; the other buffer is no longer read
+            if (row + row_step < g.d_out) issue_row(row + row_step, buf ^ 1);
+            const uint32_t* in = reinterpret_cast<const uint32_t*>(stage + buf * a.stage_bytes);
+            f32x2 P[4][4];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            if (live[r]) {
-                const uint32_t* w = in + w0s[r];
-                const uint32_t lo = w[0], mid = w[1], hi = w[2];
-                // bits [sh, sh+64) of (hi:mid:lo) as two words; pairs 0,1 come from the first word,
-                // pairs 2,3 from the 32 bits that start 2B further on (4B <= 48)
-                const uint32_t a0 = __funnelshift_r(lo, mid, shs[r]), a1 = __funnelshift_r(mid, hi, shs[r]);
-                const uint32_t b0 = __funnelshift_r(a0, a1, 2 * B);
-                const uint32_t id[4] = {a0 & mask, (a0 >> B) & mask, b0 & mask, (b0 >> B) & mask};
+            for (int r = 0; r < 4; ++r) {
+                if (FULL || live[r]) {
+                    const uint32_t* w = in + w0s[r];
+                    const uint32_t lo = w[0], mid = w[1], hi = w[2];
+                    // bits [sh, sh+64) of (hi:mid:lo) as two words; pairs 0,1 come from the first word,
+                    // pairs 2,3 from the 32 bits that start 2B further on (4B <= 48)
+                    const uint32_t a0 = __funnelshift_r(lo, mid, shs[r]), a1 = __funnelshift_r(mid, hi, shs[r]);
+                    const uint32_t b0 = __funnelshift_r(a0, a1, 2 * B);
+                    const uint32_t id[4] = {a0 & mask, (a0 >> B) & mask, b0 & mask, (b0 >> B) & mask};
 #pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    // pairs past the end of a row whose length is not a multiple of 8 have scale 0
-                    const float2 c = lds_f32x2(cb + id[p] * cb_stride);
-                    P[r][p] = pack2(c.x * sg[r][p], c.y * sg[r][p]);
+                    for (int p = 0; p < 4; ++p) {
+                        // pairs past the end of a row whose length is not a multiple of 8 have scale 0
+                        const float2 c = lds_f32x2(cb + id[p] * cb_stride);
+                        P[r][p] = pack2(c.x * sg[r][p], c.y * sg[r][p]);
+                    }
+                } else {
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) P[r][p] = pack2(0.f, 0.f);
                 }
-            } else {
+            }
+            fwht_regs<LOG2B_T, true>(P, g.log2b, tid_g);  // stage h = 1 is already in the stored codewords
+            const f32x2 rn2 = pack2(rn, rn);
 #pragma unroll
-                for (int p = 0; p < 4; ++p) P[r][p] = pack2(0.f, 0.f);
+            for (int r = 0; r < 4; ++r) {
+                const int e0 = e_out[r];
+                if (e0 >= g.d_in) continue;
+                __nv_bfloat16* dst = a.out + row * g.d_in + e0;
+                uint32_t w[4];
+                float y[8];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    unpack2(mul2(P[r][i], mul2(mcol[r][i], rn2)), y[2 * i], y[2 * i + 1]);
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
+                    w[i] = *reinterpret_cast<uint32_t*>(&h2);
+                }
+                if (FULL || g.vec) {
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        if (e0 + e < g.d_in) dst[e] = __float2bfloat16_rn(y[e]);
+                }
             }
         }
-        fwht_regs<LOG2B_T, true>(P, g.log2b, tid_g);  // stage h = 1 is already in the stored codewords
-        const f32x2 rn2 = pack2(rn, rn);
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int e0 = e_out[r];
-            if (e0 >= g.d_in) continue;
-            __nv_bfloat16* dst = a.out + row * g.d_in + e0;
-            uint32_t w[4];
-            float y[8];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                unpack2(mul2(P[r][i], mul2(mcol[r][i], rn2)), y[2 * i], y[2 * i + 1]);
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
-                w[i] = *reinterpret_cast<uint32_t*>(&h2);
-            }
-            if (g.vec) {
-                *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
-            } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    if (e0 + e < g.d_in) dst[e] = __float2bfloat16_rn(y[e]);
-            }
-        }
-    }
+    };
+    // block-uniform, so that a block runs one loop body only (two bodies in flight cost more in
+    // instruction fetch than the tests save)
+    if (g.vec) rows(std::true_type{});
+    else rows(std::false_type{});
 }
 
 // ---------------------------------------------------------------------------------------------
