@@ -1154,7 +1154,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const int e0 = e_out[r];
-                if (e0 >= g.d_in) continue;
+                if (!FULL && e0 >= g.d_in) continue;
                 __nv_bfloat16* dst = a.out + row * g.d_in + e0;
                 uint32_t w[4];
                 float y[8];
@@ -1164,7 +1164,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) decode_kernel(const DecodeArgs
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
                     w[i] = *reinterpret_cast<uint32_t*>(&h2);
                 }
-                if (FULL || g.vec) {
+                if (FULL) {  // octets beyond the row are computed like the others and not stored
+                    if (e0 < g.d_in) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+                } else if (g.vec) {
                     *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
                 } else {
 #pragma unroll
