@@ -568,9 +568,15 @@ __device__ __forceinline__ int search_overflow(const SearchSmem& s, uint2 rec, f
     return arg;
 }
 
-// Table search for a point known to lie inside the table's reach (|z| < 16000; a NaN coordinate
-// is clamped like a large one and gets some index).
-__device__ __forceinline__ int search_cell(const SearchSmem& s, float zx, float zy) {
+// A cell record whose first field is 0xFFFF points to an overflow list: {0xFFFF, offset, count, 0}.
+__device__ __forceinline__ bool cell_overflows(uint2 rec) { return (rec.x & 0xffffu) == 0xffffu; }
+
+// Nearest of the four candidates in the record of the point's cell, for a point inside the table's
+// reach (|z| < 16000; a NaN coordinate is clamped like a large one and gets some index).  There is
+// no branch in here, so that the searches of the four points of an octet interleave: the fields are
+// masked to valid indices, and the caller tests the record it gets back with cell_overflows() and
+// runs search_overflow() for such a cell (whose masked fields gave a meaningless result).
+__device__ __forceinline__ int search_cell(const SearchSmem& s, float zx, float zy, uint2& rec_out) {
     // Column and row: c = clamp(z, +-zmax), half + rn(c (c0 + t (c1 + t c2))), t = c^2, both axes in
     // packed arithmetic.  The last fused multiply-add lands on 1.5 * 2^23 + half, where the spacing
     // of f32 is 1: its rounding is the rounding to an integer, and the integer sits in the low
@@ -585,9 +591,9 @@ __device__ __forceinline__ int search_cell(const SearchSmem& s, float zx, float 
     unpack2(v, vx, vy);
     const uint32_t bx = __float_as_uint(vx), by = __float_as_uint(vy);
     const uint2 rec = lds_u32x2(s.cells + ((by * s.grid + bx) << 3));
-    const int k0 = int(rec.x & 0xffffu);
-    if (k0 == 0xffff) return search_overflow(s, rec, zx, zy);
-    const int k1 = int(rec.x >> 16), k2 = int(rec.y & 0xffffu), k3 = int(rec.y >> 16);
+    rec_out = rec;
+    const uint32_t km = uint32_t(s.K - 1);  // K is a power of two
+    const int k0 = int(rec.x & km), k1 = int((rec.x >> 16) & km), k2 = int(rec.y & km), k3 = int((rec.y >> 16) & km);
     // The list is ascending and padded by repeating its last entry (a repeated slot cannot win).
     const float2 c0 = codeword(s, k0), c1 = codeword(s, k1), c2 = codeword(s, k2), c3 = codeword(s, k3);
     const float d0 = dist2(c0, zx, zy), d1 = dist2(c1, zx, zy), d2 = dist2(c2, zx, zy), d3 = dist2(c3, zx, zy);
@@ -601,7 +607,9 @@ __device__ __forceinline__ int search_cell(const SearchSmem& s, float zx, float 
 __device__ __noinline__ int search_table(const SearchSmem& s, float zx, float zy) {
     // beyond the table's reach (or NaN): exhaustive scan
     if (!(fmaxf(fabsf(zx), fabsf(zy)) < 16000.0f)) return search_exhaustive(s, zx, zy);
-    return search_cell(s, zx, zy);
+    uint2 rec;
+    const int v = search_cell(s, zx, zy, rec);
+    return cell_overflows(rec) ? search_overflow(s, rec, zx, zy) : v;
 }
 
 // Index staging: the 4 indices of an octet are staged as one 64-bit value (index p at bits
@@ -802,12 +810,26 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                 const int k0 = 4 * Layout<LOG2B_T>::octet_after(tid_g, rr);
                 if (k0 >= n_pairs) continue;
                 uint32_t v[4];
+                if (MODE == 0) {
+                    uint2 rec[4];
+                    float2 z[4];
 #pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    const float2 z = zst[(rr * 4 + p) * 32];
-                    if (MODE == 2) v[p] = uint32_t(search_exhaustive(s, z.x, z.y));
-                    else if (MODE == 1) v[p] = uint32_t(search_table(s, z.x, z.y));
-                    else v[p] = uint32_t(search_cell(s, z.x, z.y));
+                    for (int p = 0; p < 4; ++p) {
+                        z[p] = zst[(rr * 4 + p) * 32];
+                        v[p] = uint32_t(search_cell(s, z[p].x, z[p].y, rec[p]));
+                    }
+                    // rare: one of the four cells has more than four candidates
+                    if (cell_overflows(rec[0]) || cell_overflows(rec[1]) || cell_overflows(rec[2]) || cell_overflows(rec[3])) {
+#pragma unroll
+                        for (int p = 0; p < 4; ++p)
+                            if (cell_overflows(rec[p])) v[p] = uint32_t(search_overflow(s, rec[p], z[p].x, z[p].y));
+                    }
+                } else {
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        const float2 z = zst[(rr * 4 + p) * 32];
+                        v[p] = uint32_t(MODE == 2 ? search_exhaustive(s, z.x, z.y) : search_table(s, z.x, z.y));
+                    }
                 }
                 // two indices fit a 32-bit word (B <= 12)
                 unsigned long long packed4 =
