@@ -695,11 +695,6 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
     unsigned long long* oct_s =
         reinterpret_cast<unsigned long long*>(table + table_pad) + size_t(threadIdx.x >> 5) * kStageSlotsPerWarp;
 
-    // lane-private staging of the thread's sixteen points: [slot * 4 + p][lane] float2, after the index staging
-    float2* zst = reinterpret_cast<float2*>(reinterpret_cast<unsigned long long*>(table + table_pad) +
-                                            size_t(blockDim.x >> 5) * kStageSlotsPerWarp) +
-                  size_t(threadIdx.x >> 5) * 512 + lane;
-
     f32x2 t[4][4];
     col_factors(craw, t);
     // q_k = f32(1 / (double)sigma_k): the correctly rounded f32 reciprocal is the same number (the
@@ -793,29 +788,28 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
             }
             gn = __shfl_sync(kFull, gn, 0);
             const f32x2 gn2 = pack2(gn, gn);
-            // The sixteen points of the thread go through a lane-private piece of shared memory, so
-            // that the search exists once in the instruction stream: a fully unrolled row loop does
-            // not fit the instruction cache, and fetch stalls then cost more than the extra
-            // shared-memory round trip.
+            // The sixteen points of the thread stay in the registers of the rotation.  The search loop
+            // below is rolled (a fully unrolled row loop does not fit the instruction cache, and fetch
+            // stalls then cost more than anything else), so it always works on slot 0 and the other
+            // slots move down by one after every octet.
 #pragma unroll
             for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {
                     float yx, yy;
                     unpack2(mul2(P[rr][p], gn2), yx, yy);
-                    zst[(rr * 4 + p) * 32] = make_float2(__fmul_rn(yx, q[rr][p]), __fmul_rn(yy, q[rr][p]));
+                    P[rr][p] = pack2(__fmul_rn(yx, q[rr][p]), __fmul_rn(yy, q[rr][p]));
                 }
 #pragma unroll 1
             for (int rr = 0; rr < 4; ++rr) {
                 const int k0 = 4 * Layout<LOG2B_T>::octet_after(tid_g, rr);
-                if (k0 >= n_pairs) continue;
                 uint32_t v[4];
                 if (MODE == 0) {
                     uint2 rec[4];
                     float2 z[4];
 #pragma unroll
                     for (int p = 0; p < 4; ++p) {
-                        z[p] = zst[(rr * 4 + p) * 32];
+                        unpack2(P[0][p], z[p].x, z[p].y);
                         v[p] = uint32_t(search_cell(s, z[p].x, z[p].y, rec[p]));
                     }
                     // rare: one of the four cells has more than four candidates
@@ -827,15 +821,24 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                 } else {
 #pragma unroll
                     for (int p = 0; p < 4; ++p) {
-                        const float2 z = zst[(rr * 4 + p) * 32];
+                        float2 z;
+                        unpack2(P[0][p], z.x, z.y);
                         v[p] = uint32_t(MODE == 2 ? search_exhaustive(s, z.x, z.y) : search_table(s, z.x, z.y));
                     }
                 }
                 // two indices fit a 32-bit word (B <= 12)
                 unsigned long long packed4 =
                     (unsigned long long)(v[0] | (v[1] << B)) | ((unsigned long long)(v[2] | (v[3] << B)) << (2 * B));
-                if (k0 + 4 > n_pairs) packed4 &= (1ull << ((n_pairs - k0) * B)) - 1ull;  // the row ends inside this octet
-                oct_s[stage_slot((k0 >> 2) - oct0)] = packed4;
+                if (k0 < n_pairs) {
+                    if (k0 + 4 > n_pairs) packed4 &= (1ull << ((n_pairs - k0) * B)) - 1ull;  // the row ends inside this octet
+                    oct_s[stage_slot((k0 >> 2) - oct0)] = packed4;
+                }
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {  // next octet into slot 0
+                    P[0][p] = P[1][p];
+                    P[1][p] = P[2][p];
+                    P[2][p] = P[3][p];
+                }
             }
             __syncwarp();
             // bit packing of the warp's segment: octet o occupies bits [o*4B, (o+1)*4B) (LSB first)
@@ -1490,11 +1493,11 @@ extern "C" int qamw_codebook_create(const float* codebook_host, int K, int grid,
     if (grid < 0 || grid > 255 || (grid > 0 && grid % 2 == 0)) return QAMW_ERR_ARG;
     *out = nullptr;
     SearchTable t;
-    // The encoder's shared memory also holds 84 KB of per-warp staging (16 warps x (1.25 KB of
-    // indices + 4 KB of points)) and the codebook in four bank-separated copies (one copy for
-    // K = 4096): the table gets what is left of the 227 KB of one SM.  The grid side is odd.
-    const size_t copies = K <= 2048 ? 4 : 1;
-    const size_t budget = kSmemLimit - kEncodeStaticSmem - size_t(16) * (kStageSlotsPerWarp * 8 + 512 * 8) - size_t(K) * 8 * copies;
+    // The encoder's shared memory also holds 20 KB of per-warp index staging (16 warps x 1.25 KB)
+    // and the codebook in eight bank-separated copies (two for K = 4096): the table gets what is left
+    // of the 227 KB of one SM.  The grid side is odd.
+    const size_t copies = K <= 2048 ? 8 : 2;
+    const size_t budget = kSmemLimit - kEncodeStaticSmem - size_t(16) * (kStageSlotsPerWarp * 8) - size_t(K) * 8 * copies;
     if (!choose_search_table(codebook_host, K, grid, budget, &t)) return QAMW_ERR_NOMEM;
     qamw_codebook* cb = new (std::nothrow) qamw_codebook();
     if (!cb) return QAMW_ERR_NOMEM;
@@ -1579,7 +1582,7 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     a.row_norm = row_norm_out;
     a.inv_sqrt_b = float(1.0 / std::sqrt(double(p->block)));
     const size_t fixed = ((size_t(a.table_bytes) + 15) & ~size_t(15)) +
-                         size_t(a.g.groups) * (a.g.tg / 32) * (kStageSlotsPerWarp * 8 + 512 * 8);
+                         size_t(a.g.groups) * (a.g.tg / 32) * (kStageSlotsPerWarp * 8);
     if (fixed + size_t(p->K) * 8 > kSmemLimit - kEncodeStaticSmem) return QAMW_ERR_NOMEM;
     a.log2c = pick_log2_copies(p->K, kSmemLimit - kEncodeStaticSmem - fixed);
     const size_t smem = fixed + (size_t(p->K) * 8 << a.log2c);
