@@ -788,10 +788,9 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
             }
             gn = __shfl_sync(kFull, gn, 0);
             const f32x2 gn2 = pack2(gn, gn);
-            // The sixteen points of the thread stay in the registers of the rotation.  The search loop
-            // below is rolled (a fully unrolled row loop does not fit the instruction cache, and fetch
-            // stalls then cost more than anything else), so it always works on slot 0 and the other
-            // slots move down by one after every octet.
+            // The sixteen points of the thread stay in the registers of the rotation; the search is
+            // unrolled over the four octets (the branch-free search is compact enough for that: with a
+            // branch per point the unrolled loop did not fit the instruction cache).
 #pragma unroll
             for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
@@ -800,7 +799,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                     unpack2(mul2(P[rr][p], gn2), yx, yy);
                     P[rr][p] = pack2(__fmul_rn(yx, q[rr][p]), __fmul_rn(yy, q[rr][p]));
                 }
-#pragma unroll 1
+#pragma unroll
             for (int rr = 0; rr < 4; ++rr) {
                 const int k0 = 4 * Layout<LOG2B_T>::octet_after(tid_g, rr);
                 uint32_t v[4];
@@ -809,7 +808,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                     float2 z[4];
 #pragma unroll
                     for (int p = 0; p < 4; ++p) {
-                        unpack2(P[0][p], z[p].x, z[p].y);
+                        unpack2(P[rr][p], z[p].x, z[p].y);
                         v[p] = uint32_t(search_cell(s, z[p].x, z[p].y, rec[p]));
                     }
                     // rare: one of the four cells has more than four candidates
@@ -822,7 +821,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
 #pragma unroll
                     for (int p = 0; p < 4; ++p) {
                         float2 z;
-                        unpack2(P[0][p], z.x, z.y);
+                        unpack2(P[rr][p], z.x, z.y);
                         v[p] = uint32_t(MODE == 2 ? search_exhaustive(s, z.x, z.y) : search_table(s, z.x, z.y));
                     }
                 }
@@ -832,12 +831,6 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                 if (k0 < n_pairs) {
                     if (k0 + 4 > n_pairs) packed4 &= (1ull << ((n_pairs - k0) * B)) - 1ull;  // the row ends inside this octet
                     oct_s[stage_slot((k0 >> 2) - oct0)] = packed4;
-                }
-#pragma unroll
-                for (int p = 0; p < 4; ++p) {  // next octet into slot 0
-                    P[0][p] = P[1][p];
-                    P[1][p] = P[2][p];
-                    P[2][p] = P[3][p];
                 }
             }
             __syncwarp();
