@@ -23,11 +23,12 @@
 //     bank conflicts), hence: the codebook is stored in several bank-separated copies and every
 //     lane reads the copy of its own banks.
 //   * A warp owns 1024 consecutive elements: whole Hadamard blocks and 64*B consecutive bytes of
-//     the packed row.  The encoder (whose row norms come from a kernel of their own) and the
-//     decoder therefore have no barrier after their prologue; each warp stages its own piece of
-//     the packed row in shared memory.
-//   * The encoder's search exists once in its instruction stream (a rolled loop fed from a
-//     lane-private staging area): sixteen inlined copies per row overflow the instruction cache.
+//     the packed row.  The decoder therefore has no barrier after its prologue, and the warps of
+//     an encoder row meet once per row, for the row norm; each warp stages its own piece of the
+//     packed row in shared memory.
+//   * The encoder's four-candidate search has no branch, so that the sixteen searches of a thread
+//     (unrolled) interleave; the kernel is sensitive to the size of that loop body, which is why
+//     the rare paths (overflow lists, reach check, exhaustive scan) are kept out of it.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
