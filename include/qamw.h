@@ -59,6 +59,10 @@ extern "C" {
                                     different streams run side by side and each one's start-up (tables and
                                     per-column constants into shared memory and registers) hides behind the other */
 
+#define QAMW_FLAG_GENERAL_KERNELS 4u /* encode, decode: always run the general row kernels (any d_in, any alignment, any
+                                       block size), also where the faster kernels for the common layouts would apply;
+                                       same results, meant for testing */
+
 #define QAMW_DEFAULT_SIGN_SEED 0x51A5C0DEC0FFEE01ULL
 #define QAMW_MAX_BLOCK 1024 /* cap of Section 3.3 */
 #define QAMW_MAX_K 4096

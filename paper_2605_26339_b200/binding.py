@@ -22,6 +22,7 @@ ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_CUDA, ERR_NONFINITE, ERR_NOMEM = -1, -2, -3, 
 DTYPE_F32, DTYPE_BF16 = 0, 1
 FLAG_BRUTE_FORCE = 1
 FLAG_HALF_DEVICE = 2
+FLAG_GENERAL_KERNELS = 4
 DEFAULT_SIGN_SEED = 0x51A5C0DEC0FFEE01
 _ERR_NAMES = {-1: "QAMW_ERR_ARG", -2: "QAMW_ERR_SHAPE", -3: "QAMW_ERR_ALIGN", -4: "QAMW_ERR_CUDA",
               -5: "QAMW_ERR_NONFINITE", -6: "QAMW_ERR_NOMEM"}

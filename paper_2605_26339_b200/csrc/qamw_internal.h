@@ -76,6 +76,32 @@ bool pack_search_table(const CellLists& cl, SearchTable* out);
 bool choose_search_table(const float* codebook, int K, int grid, size_t budget_bytes, SearchTable* out);
 
 void set_cuda_error(const char* what, int code);
+void set_error_text(const char* text);
+
+// One weight matrix as the batched (multi-matrix) kernels see it: plain device pointers and sizes.
+struct MatDesc {
+    const void* W;
+    const float* chan_scale;
+    const int8_t* signs;
+    const float* sigma;
+    const float* act_rms;
+    uint8_t* packed;
+    float* row_norm;
+    void* w_hat;
+    double* dist4;
+    long long w_row_stride;       // elements
+    long long packed_row_stride;  // bytes
+    int d_out, d_in;
+};
+
+// Fast multi-matrix paths (qamw_rows.cu).  `descs` is a device array of n descriptors, or NULL with
+// n == 1 and the single descriptor passed by value.  They return QAMW_ERR_SHAPE without launching
+// when a matrix does not meet the fast kernels' layout rules; the caller then uses the general kernels.
+int rows_decode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, int block, int K,
+                const float* codebook_dev, uint32_t flags, void* stream);
+int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, int block, int K, int w_bf16,
+                const struct ::qamw_codebook* cb, uint32_t flags, int32_t* status, void* stream);
+int sm_count();
 
 }  // namespace qamw
 
