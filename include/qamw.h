@@ -220,6 +220,52 @@ int qamw_decode(const uint8_t* packed, const float* row_norm, const float* chan_
 int qamw_distortion(const void* W, const void* w_hat_bf16, const float* act_rms, const qamw_params* p,
                     double* out4, void* stream);
 
+/* ----------------------------------------------------------------------------------------------
+ * Batches: every linear weight of a layer or of a whole model behind one handle, so that one
+ * persistent launch per phase walks all matrices (Section 3.1 / 3.2 applied matrix after matrix,
+ * as the paper's quantisation driver does).  The shared-memory tables are then filled once per
+ * phase instead of once per matrix, which is what small matrices spend their time on otherwise.
+ * -------------------------------------------------------------------------------------------- */
+
+/* One matrix of a batch: the arguments of the single-matrix entry points, all device pointers.
+ * chan_scale and act_rms may be NULL; a pointer that a phase does not use may be NULL as long as
+ * that phase is never called on the batch (e.g. no W for a decode-only batch). */
+typedef struct {
+    qamw_params p;
+    const void* W;           /* [d_out, w_row_stride] f32 or bf16 */
+    const float* chan_scale; /* [d_in] or NULL */
+    const int8_t* signs;     /* [d_in] */
+    float* sigma;            /* [d_in/2]: written by qamw_calibrate_batch, read by encode and decode */
+    const float* act_rms;    /* [d_in] or NULL: weights of the distortion sums */
+    uint8_t* packed;         /* [d_out, packed_row_stride] */
+    float* row_norm;         /* [d_out] */
+    void* w_hat_bf16;        /* [d_out, d_in] bf16 */
+    double* dist4;           /* 4 doubles */
+} qamw_matrix;
+
+typedef struct qamw_batch qamw_batch; /* opaque: validated copy of the items plus their device descriptors */
+
+/* Validates n items (host array, copied) against the rules of the single-matrix calls and uploads
+ * their descriptors to the current device, which must be the codebook's.  All items share block, K
+ * and w_dtype (QAMW_ERR_ARG otherwise).  Synchronous; allocates n small descriptors on the device,
+ * released by qamw_batch_destroy.  The codebook must outlive the batch. */
+int qamw_batch_create(const qamw_matrix* items, int n, const qamw_codebook* cb, qamw_batch** out);
+void qamw_batch_destroy(qamw_batch* b);
+
+/* Device scratch qamw_calibrate_batch needs (the per-matrix needs, each rounded up to 256 bytes). */
+size_t qamw_batch_workspace_bytes(const qamw_batch* b);
+
+/* The four phases over all matrices of the batch, each equivalent to calling the single-matrix
+ * entry point on every item in order (same results bit for bit, same error codes), asynchronous on
+ * `stream`.  Matrices in the common layout (rows and metadata 16-byte aligned, d_in a multiple of
+ * 16, block >= 32) are handled by one launch per phase; if any item falls outside, the phase falls
+ * back to one launch per matrix. */
+int qamw_calibrate_batch(const qamw_batch* b, void* workspace, size_t workspace_bytes, int32_t* status_out,
+                         void* stream);
+int qamw_encode_batch(const qamw_batch* b, int32_t* status_out, void* stream);
+int qamw_decode_batch(const qamw_batch* b, void* stream);
+int qamw_distortion_batch(const qamw_batch* b, void* stream);
+
 /* Last CUDA error string seen by the library on this thread (host, static storage). */
 const char* qamw_last_cuda_error(void);
 

@@ -33,6 +33,8 @@ EXPORTED = [
     "qamw_codebook_destroy", "qamw_codebook_table_info", "qamw_search_table_build",
     "qamw_calibrate_workspace_bytes", "qamw_calibrate", "qamw_calibrate_static", "qamw_encode", "qamw_rotate", "qamw_decode",
     "qamw_distortion", "qamw_last_cuda_error",
+    "qamw_batch_create", "qamw_batch_destroy", "qamw_batch_workspace_bytes", "qamw_calibrate_batch",
+    "qamw_encode_batch", "qamw_decode_batch", "qamw_distortion_batch",
 ]
 
 
@@ -46,6 +48,13 @@ class Params(C.Structure):
     _fields_ = [("d_out", C.c_int32), ("d_in", C.c_int32), ("block", C.c_int32), ("K", C.c_int32),
                 ("w_dtype", C.c_int32), ("flags", C.c_uint32), ("w_row_stride", C.c_int64),
                 ("packed_row_stride", C.c_int64)]
+
+
+class Matrix(C.Structure):
+    """qamw_matrix: one weight matrix of a batch (device pointers)."""
+    _fields_ = [("p", Params), ("W", C.c_void_p), ("chan_scale", C.c_void_p), ("signs", C.c_void_p),
+                ("sigma", C.c_void_p), ("act_rms", C.c_void_p), ("packed", C.c_void_p), ("row_norm", C.c_void_p),
+                ("w_hat_bf16", C.c_void_p), ("dist4", C.c_void_p)]
 
 
 _lib = None
@@ -84,6 +93,15 @@ def lib() -> C.CDLL:
         L.qamw_decode.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_distortion.argtypes = [vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_last_cuda_error.restype = C.c_char_p
+        L.qamw_batch_create.argtypes = [C.POINTER(Matrix), i32, vp, C.POINTER(vp)]
+        L.qamw_batch_destroy.argtypes = [vp]
+        L.qamw_batch_destroy.restype = None
+        L.qamw_batch_workspace_bytes.argtypes = [vp]
+        L.qamw_batch_workspace_bytes.restype = sz
+        L.qamw_calibrate_batch.argtypes = [vp, vp, sz, vp, vp]
+        L.qamw_encode_batch.argtypes = [vp, vp, vp]
+        L.qamw_decode_batch.argtypes = [vp, vp]
+        L.qamw_distortion_batch.argtypes = [vp, vp]
         _lib = L
     return _lib
 
@@ -281,3 +299,54 @@ def decode(packed: torch.Tensor, row_norm: torch.Tensor, chan_scale, signs, sigm
 def distortion(W: torch.Tensor, w_hat: torch.Tensor, act_rms, p: Params, out4: torch.Tensor, stream=None):
     _check("qamw_distortion", lib().qamw_distortion(_dp(W), _dp(w_hat), _dp(act_rms), C.byref(p), _dp(out4),
                                                    _stream(stream)))
+
+
+# ------------------------------------------------------------------------------- batches
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def make_matrix(p: Params, W=None, chan_scale=None, signs=None, sigma=None, act_rms=None, packed=None,
+                row_norm=None, w_hat=None, dist4=None) -> Matrix:
+    """qamw_matrix from torch tensors (device); the caller keeps the tensors alive."""
+    return Matrix(p, _ptr(W), _ptr(chan_scale), _ptr(signs), _ptr(sigma), _ptr(act_rms), _ptr(packed),
+                  _ptr(row_norm), _ptr(w_hat), _ptr(dist4))
+
+
+class Batch:
+    """Owns a qamw_batch* (all matrices of a layer or model) on the current CUDA device."""
+
+    def __init__(self, matrices, cb: Codebook):
+        self.n = len(matrices)
+        arr = (Matrix * self.n)(*matrices)
+        self._cb = cb  # the codebook must outlive the batch
+        h = C.c_void_p()
+        _check("qamw_batch_create", lib().qamw_batch_create(arr, self.n, cb.handle, C.byref(h)))
+        self._h = h
+
+    def workspace_bytes(self) -> int:
+        return int(lib().qamw_batch_workspace_bytes(self._h))
+
+    def calibrate(self, workspace: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None):
+        _check("qamw_calibrate_batch", lib().qamw_calibrate_batch(
+            self._h, _dp(workspace), workspace.numel() * workspace.element_size(), _dp(status), _stream(stream)))
+
+    def encode(self, status: Optional[torch.Tensor] = None, stream=None):
+        _check("qamw_encode_batch", lib().qamw_encode_batch(self._h, _dp(status), _stream(stream)))
+
+    def decode(self, stream=None):
+        _check("qamw_decode_batch", lib().qamw_decode_batch(self._h, _stream(stream)))
+
+    def distortion(self, stream=None):
+        _check("qamw_distortion_batch", lib().qamw_distortion_batch(self._h, _stream(stream)))
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().qamw_batch_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

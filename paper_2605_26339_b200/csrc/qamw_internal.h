@@ -97,11 +97,12 @@ struct MatDesc {
 // Fast multi-matrix paths (qamw_rows.cu).  `descs` is a device array of n descriptors, or NULL with
 // n == 1 and the single descriptor passed by value.  They return QAMW_ERR_SHAPE without launching
 // when a matrix does not meet the fast kernels' layout rules; the caller then uses the general kernels.
-int rows_decode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, int block, int K,
-                const float* codebook_dev, uint32_t flags, void* stream);
-int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, int block, int K, int w_bf16,
-                const struct ::qamw_codebook* cb, uint32_t flags, int32_t* status, void* stream);
+int rows_decode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, const void* spans_dev, int span_blocks,
+                int block, int K, const float* codebook_dev, uint32_t flags, void* stream);
+int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, const void* spans_dev, int span_blocks,
+                int block, int K, int w_bf16, const ::qamw_codebook* cb, uint32_t flags, int32_t* status, void* stream);
 int sm_count();
+int check_matrix_params(const qamw_params* p);  // QAMW_OK or the error code every entry point reports
 
 }  // namespace qamw
 

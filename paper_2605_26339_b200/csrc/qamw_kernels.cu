@@ -1209,6 +1209,10 @@ int launch_decode(const DecodeArgs& a, int blocks, size_t smem, cudaStream_t st)
 
 }  // namespace
 
+namespace qamw {
+int check_matrix_params(const qamw_params* p) { return check_params(p); }
+}  // namespace qamw
+
 // ---------------------------------------------------------------------------------------------
 // C ABI
 // ---------------------------------------------------------------------------------------------
@@ -1283,6 +1287,22 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     if (p->packed_row_stride < (long long)row_bytes || p->packed_row_stride % 4) return QAMW_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(packed_out) % 4) return QAMW_ERR_ALIGN;
     if (p->d_out == 0) return QAMW_OK;
+    if (!(p->flags & QAMW_FLAG_GENERAL_KERNELS)) {  // common layouts: the multi-matrix kernel, here with one matrix
+        MatDesc d{};
+        d.W = W;
+        d.chan_scale = chan_scale;
+        d.signs = signs;
+        d.sigma = sigma;
+        d.packed = packed_out;
+        d.row_norm = row_norm_out;
+        d.w_row_stride = p->w_row_stride;
+        d.packed_row_stride = p->packed_row_stride;
+        d.d_out = p->d_out;
+        d.d_in = p->d_in;
+        rc = rows_encode(nullptr, &d, 1, nullptr, 0, p->block, p->K, p->w_dtype == QAMW_DTYPE_BF16, cb, p->flags,
+                         status_out, stream);
+        if (rc != QAMW_ERR_SHAPE) return rc;
+    }
     EncodeArgs a;
     a.g = make_geom(p, W);
     a.g.cvec = const_vec_ok(p, chan_scale, signs, sigma);
@@ -1476,7 +1496,7 @@ extern "C" int qamw_decode(const uint8_t* packed, const float* row_norm, const f
         d.packed_row_stride = p->packed_row_stride;
         d.d_out = p->d_out;
         d.d_in = p->d_in;
-        rc = rows_decode(nullptr, &d, 1, p->block, p->K, static_cast<const float*>(cb->d_blob), p->flags, stream);
+        rc = rows_decode(nullptr, &d, 1, nullptr, 0, p->block, p->K, static_cast<const float*>(cb->d_blob), p->flags, stream);
         if (rc != QAMW_ERR_SHAPE) return rc;
     }
     DecodeArgs a;

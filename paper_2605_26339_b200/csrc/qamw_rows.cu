@@ -1,4 +1,4 @@
-// Row kernels of libqamw for the common layouts (16-byte aligned rows, d_in a multiple of 16,
+// Row kernels of libqamw for the common layouts (32-byte aligned rows, d_in a multiple of 16,
 // Hadamard blocks of 32 elements or more): one persistent launch walks any number of matrices.
 //
 // Geometry.
@@ -6,31 +6,37 @@
 //     per thread in the decoder, NS = 2 (16 elements) in the encoder, whose register budget then
 //     allows 20 to 28 resident warps per SM instead of 15.  A row is owned by a group of
 //     ceil(d_in / (256 NS)) warps; a block holds as many groups as fit and the grid is persistent.
-//   * A launch takes an array of matrix descriptors.  Every block walks all matrices; the tables in
-//     shared memory (codebook copies, cell records) are filled once per launch, and only the
-//     per-column constants of a warp's segment are reloaded when the matrix changes.
+//   * A launch takes an array of matrix descriptors.  The rows of all matrices form one list, cut
+//     into one contiguous span per block with (nearly) equal numbers of weights, so a block meets one
+//     or two matrices; the tables in shared memory (codebook copies, cell records) are filled once
+//     per launch and only the per-column constants of a warp's segment are reloaded when the matrix
+//     changes.
 //   * Walsh-Hadamard butterflies of a block of b elements: stages h = 1, 2, 4 inside an octet, then
 //     one stage per octet slot bit inside the thread, then one "half exchange" per lane bit: a thread
 //     keeps the slots whose top slot bit is 0, sends the others to its partner (lane ^ 2^j), and
 //     computes both outputs (K + R, K - R) of the butterflies whose inputs it then holds.  Every
 //     exchange uses the top slot bit, so after the last stage a thread holds runs of NS/2 adjacent
 //     octets and the threads of a block cover consecutive runs: 32-byte stores that tile full
-//     128-byte lines (decoder).  Which physical slot receives the sum and which the difference is
-//     chosen so that the next stage can again keep slot 0 and send slot 1 without moving registers;
-//     for threads that need the other placement the received value is multiplied by -1 first
-//     (K - R, K + R).  An upper partner then holds R - K as K - R: some slots end up negated, by
-//     a pattern that depends on the lane only and is folded into the per-column constants.
-//     Stages run in ascending order of h with one f32 rounding per output, and a multiplication by
-//     +-1 is exact, so the result is bit-identical to the plain butterfly.
+//     128-byte lines (decoder).  A thread starts with NS consecutive octets.  Which physical slot
+//     receives the sum and which the difference of a stage is chosen so that the next stage can again
+//     keep the lower slots and send the upper ones without moving registers: a thread whose next lane
+//     bit is set multiplies the received value by -1 first (K - R, K + R), and the last in-thread
+//     stage does the same for odd lanes.  An upper partner then holds R - K as K - R: some slots end
+//     up negated, by a pattern that depends on the lane only and is folded into the per-column
+//     constants.  Stages run in ascending order of h with one f32 rounding per output, and a
+//     multiplication by +-1 is exact, so the result is bit-identical to the plain butterfly.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <mutex>
+#include <new>
 #include <type_traits>
 #include <unordered_map>
+#include <vector>
 
 #include "qamw_device.cuh"
 #include "qamw_internal.h"
@@ -51,10 +57,8 @@ struct Lay2 {
     static_assert(S >= 0 && S <= 5, "block size out of range for this geometry");
     static constexpr int L = 1 << S;
     // octet (units of 8 elements, relative to the warp's segment) in physical slot p before the
-    // butterflies: NS consecutive octets per lane; odd lanes hold the two halves swapped
-    __device__ static __forceinline__ int octet_before(int lane, int p) {
-        return NS * lane + (S >= 1 ? (p ^ (TOP * (lane & 1))) : p);
-    }
+    // butterflies: NS consecutive octets per lane
+    __device__ static __forceinline__ int octet_before(int lane, int p) { return NS * lane + p; }
     // ... and after them
     __device__ static __forceinline__ int octet_after(int lane, int p) {
         if (S == 0) return NS * lane + p;
@@ -112,8 +116,9 @@ __device__ __forceinline__ void fwht2(f32x2 (&P)[NS][4], int lane) {
             bfly2(P[2 % NS][i], P[3 % NS][i]);
         }
     }
-    // top slot bit (h = 8 for NS = 2, h = 16 for NS = 4).  An odd lane holds its halves swapped, so
-    // its sum and difference change places: out_lo = s lo + hi, out_hi = lo - s hi with s = -1.
+    // top slot bit (h = 8 for NS = 2, h = 16 for NS = 4).  The first half exchange wants the two
+    // halves of an odd lane in swapped places, so an odd lane writes its difference into the lower
+    // slots and its sum into the upper ones: out_lo = a + s c, out_hi = a - s c with s = -1.
     if (Lay::S >= 1) {
         const float s0 = (lane & 1) ? -1.0f : 1.0f;
         const f32x2 sp = pack2(s0, s0), sn = pack2(-s0, -s0);
@@ -122,7 +127,7 @@ __device__ __forceinline__ void fwht2(f32x2 (&P)[NS][4], int lane) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const f32x2 a = P[p][i], c = P[p + TOP][i];
-                P[p][i] = fma2(a, sp, c);
+                P[p][i] = fma2(c, sp, a);
                 P[p + TOP][i] = fma2(c, sn, a);
             }
     } else {
@@ -165,10 +170,23 @@ __device__ __forceinline__ void st_global_256(void* p, const uint32_t (&w)[8]) {
                  "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
                  : "memory");
 }
+__device__ __forceinline__ void ld_global_256(const void* p, uint32_t (&w)[8]) {
+    asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p));
+}
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
+}
+
+// The span of the concatenated row list that this block works on: first matrix, first row in it,
+// last matrix, end row in it.  Without a span table there is one matrix, split evenly.
+__device__ __forceinline__ int4 block_span(const int4* spans, int d_out_single) {
+    if (spans) return spans[blockIdx.x];
+    const long long n = d_out_single;
+    return make_int4(0, int(n * blockIdx.x / gridDim.x), 0, int(n * (blockIdx.x + 1) / gridDim.x));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -177,11 +195,11 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
 struct Decode2Args {
     const MatDesc* descs;    // device array, or NULL: `one` is the only matrix
     MatDesc one;
-    int n_mats;
+    const int4* spans;       // per block (see block_span), or NULL
     const float2* codebook;  // device, K entries
     int K, log2K, log2c;
     int seg_bytes;           // packed bytes of one warp segment: 16 * NS * B
-    int stage_bytes;         // one staging buffer of a warp: seg_bytes + 16
+    int stage_bytes;         // one staging buffer of a warp (128-byte aligned, at least seg_bytes + 16)
     float inv_sqrt_b;
 };
 
@@ -209,8 +227,8 @@ __global__ void __launch_bounds__(NS == 4 ? 512 : 896, 1) decode2_kernel(const D
     if (lane < 8) reinterpret_cast<uint32_t*>(stage + (lane >> 2) * a.stage_bytes + a.seg_bytes)[lane & 3] = 0u;
     __syncthreads();
 
-    // where this thread's index bits sit inside a staged segment: two runs (physical slots with the
-    // top slot bit 0 / 1), each 4 B TOP bits long
+    // where this thread's index bits sit inside a staged segment: two runs (the lower and the upper
+    // physical slots), each 4 B TOP bits long
     uint32_t run_word[2], run_shift[2];
 #pragma unroll
     for (int x = 0; x < 2; ++x) {
@@ -219,34 +237,42 @@ __global__ void __launch_bounds__(NS == 4 ? 512 : 896, 1) decode2_kernel(const D
         run_shift[x] = bit0 & 31u;
     }
 
-    for (int m = 0; m < a.n_mats; ++m) {
+    const int4 span = block_span(a.spans, a.one.d_out);
+    for (int m = span.x; m <= span.z; ++m) {
         const MatDesc& d = a.descs ? a.descs[m] : a.one;
-        const int d_in = d.d_in, d_out = d.d_out, n_pairs = d_in >> 1;
+        const int d_in = d.d_in, n_pairs = d_in >> 1;
+        const int row_begin = m == span.x ? span.y : 0;
+        const int row_end = m == span.z ? span.w : d.d_out;
         const int n_seg = (d_in + WE - 1) / WE;
-        const int groups = n_warps / n_seg;           // >= 1 (checked on the host)
+        const int groups = n_warps / n_seg;  // >= 1 (checked on the host)
         const int group = warp / n_seg, seg = warp - group * n_seg;
-        if (group >= groups) continue;                // this warp has no segment in this matrix
-        const uint8_t* packed = d.packed;
+        const int row0 = row_begin + group;
+        if (group >= groups || row0 >= row_end) continue;  // this warp has no work in this matrix
+        const int row_step = groups;
+        const int n_rows = (row_end - row0 + row_step - 1) / row_step;
         const long long pstride = d.packed_row_stride;
         const int row_bytes = int((((long long)n_pairs * B + 7) / 8 + 15) & ~15LL);  // <= stride (a multiple of 16)
         const long long seg_off = (long long)seg * a.seg_bytes;
-        const int seg_len = max(0, min(a.seg_bytes, row_bytes - int(seg_off)));
-        const int n_chunks = seg_len >> 4;
-        auto issue_row = [&](long long row, int buf) {
-            const unsigned char* src = packed + row * pstride + seg_off;
+        const int n_chunks = max(0, min(a.seg_bytes, row_bytes - int(seg_off))) >> 4;
+        // at most 48 chunks of 16 bytes per segment: two predicated copies per lane, no loop
+        const bool copy0 = lane < n_chunks, copy1 = lane + 32 < n_chunks;
+        auto issue_row = [&](const unsigned char* src, int buf) {
             unsigned char* dst = stage + buf * a.stage_bytes;
-            for (int c = lane; c < n_chunks; c += 32) cp_async(dst + (size_t(c) << 4), src + (size_t(c) << 4), 4);
+            if (copy0) cp_async(dst + (lane << 4), src + (lane << 4), 4);
+            if (copy1) cp_async(dst + ((lane + 32) << 4), src + ((lane + 32) << 4), 4);
             cp_async_commit();
         };
-        const long long row_step = (long long)gridDim.x * groups;
-        long long row = (long long)((blockIdx.x + 17u * unsigned(m)) % gridDim.x) * groups + group;
+        const unsigned char* src = d.packed + (long long)row0 * pstride + seg_off;  // next row to fetch
+        const long long src_step = (long long)row_step * pstride;
         __syncwarp();  // the previous matrix's last row has been read by every lane
-        if (row < d_out) issue_row(row, 0);
+        issue_row(src, 0);
+        src += src_step;
 
         // per-column constants of this warp's segment
         const int oct0 = seg * (WE / 8);  // first octet of the segment
         float sg[NS][4];
         f32x2 mcol[NS][4];
+        bool store_ok[NS];
         int e_out[NS];
 #pragma unroll
         for (int p = 0; p < NS; ++p) {
@@ -254,6 +280,7 @@ __global__ void __launch_bounds__(NS == 4 ? 512 : 896, 1) decode2_kernel(const D
             load4f(d.sigma, k0, n_pairs, 1, 0.f, sg[p]);
             const int e0 = 8 * (oct0 + Lay::octet_after(lane, p));
             e_out[p] = e0;
+            store_ok[p] = e0 < d_in;
             float cs[8], sgn[8];
             if (d.chan_scale) {
                 load8f(d.chan_scale, e0, d_in, 1, 1.0f, cs);
@@ -268,15 +295,19 @@ __global__ void __launch_bounds__(NS == 4 ? 512 : 896, 1) decode2_kernel(const D
                 mcol[p][i] = pack2(fl * __fdiv_rn(sgn[2 * i] * a.inv_sqrt_b, cs[2 * i]),
                                    fl * __fdiv_rn(sgn[2 * i + 1] * a.inv_sqrt_b, cs[2 * i + 1]));
         }
-        __nv_bfloat16* out = static_cast<__nv_bfloat16*>(d.w_hat);
-        const float* row_norm = d.row_norm;
+        __nv_bfloat16* orow = static_cast<__nv_bfloat16*>(d.w_hat) + (long long)row0 * d_in;
+        const long long out_step = (long long)row_step * d_in;
+        const float* rnp = d.row_norm + row0;
 
         int buf = 0;
-        for (; row < d_out; row += row_step, buf ^= 1) {
-            const float rn = __ldg(row_norm + row);
+        for (int it = 0; it < n_rows; ++it, buf ^= 1, orow += out_step, rnp += row_step) {
+            const float rn = __ldg(rnp);
             cp_async_wait_all();
             __syncwarp();  // every lane's part of this row has landed; the other buffer is no longer read
-            if (row + row_step < d_out) issue_row(row + row_step, buf ^ 1);
+            if (it + 1 < n_rows) {
+                issue_row(src, buf ^ 1);
+                src += src_step;
+            }
             const uint32_t in = stage_addr + uint32_t(buf * a.stage_bytes);
             f32x2 P[NS][4];
 #pragma unroll
@@ -320,7 +351,6 @@ __global__ void __launch_bounds__(NS == 4 ? 512 : 896, 1) decode2_kernel(const D
             }
             fwht2<NS, LOG2B, true>(P, lane);
             const f32x2 rn2 = pack2(rn, rn);
-            __nv_bfloat16* orow = out + row * d_in;
 #pragma unroll
             for (int p = 0; p < NS; p += (NS == 4 ? 2 : 1)) {
                 constexpr int NP = NS == 4 ? 2 : 1;  // adjacent octets written by one store
@@ -334,17 +364,302 @@ __global__ void __launch_bounds__(NS == 4 ? 512 : 896, 1) decode2_kernel(const D
                         __nv_bfloat162 h2 = __floats2bfloat162_rn(y0, y1);
                         w[4 * t + i] = *reinterpret_cast<uint32_t*>(&h2);
                     }
-                const int e0 = e_out[p];
-                if (e0 < d_in) {
+                if (store_ok[p]) {
                     if constexpr (NS == 4) {
-                        st_global_256(orow + e0, w);
+                        st_global_256(orow + e_out[p], w);
                     } else {
-                        *reinterpret_cast<uint4*>(orow + e0) = make_uint4(w[0], w[1], w[2], w[3]);
+                        *reinterpret_cast<uint4*>(orow + e_out[p]) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
             }
         }
         cp_async_wait_all();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// encoder
+// ---------------------------------------------------------------------------------------------
+struct Encode2Args {
+    const MatDesc* descs;
+    MatDesc one;
+    const int4* spans;
+    const float2* codebook;  // device, K entries
+    const uint4* table;      // cells | overflow, as laid out by qamw_codebook_create
+    int table_bytes;         // a multiple of 16
+    int off_overflow;        // byte offset inside the table
+    int K, log2K, grid;
+    float map_zmax, map_c0, map_c1, map_c2, map_bias;  // the cell map of the table
+    int log2c;               // log2 of the number of codebook copies in shared memory
+    int brute;
+    float inv_sqrt_b;        // c_b = f32(1 / sqrt(b))
+    int32_t* status;         // out (optional): bit 0 set when a row norm is not finite
+};
+
+// Index staging of a warp: its 64 octets as one 64-bit value each (index p of the octet at bits
+// [p B, (p+1) B)); 8 slots of padding after every 16 keep the two stores of a warp on distinct banks
+// for the common block sizes.
+template <int NS>
+struct Stage2 {
+    static constexpr int kSlots = NS == 2 ? 96 : 160;  // 32 NS octets plus their padding
+    __device__ static __forceinline__ int slot(int o) { return NS == 2 ? o + ((o >> 4) << 3) : o + ((o >> 4) << 2); }
+};
+
+// Encoder, two octets per thread.  A warp owns 512 consecutive elements of a row: it scales them,
+// adds up its part of the row norm, rotates (shuffles only), and after the one meeting point of the
+// row's warps -- a named barrier for the norm -- searches its 256 pairs, stages the indices and
+// writes its 32 B bytes of the packed row.  W is read once.
+template <bool BF16, int LOG2B, int NS, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
+    constexpr int WE = 256 * NS;
+    typedef Lay2<NS, LOG2B> Lay;
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ double ss_part[2][32];  // per-warp partial sums of squares, two rows in flight
+    __shared__ MatDesc cur;            // the matrix the block is working on (re-read per row: saves registers)
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+
+    const int cb_bytes = (a.K * 8) << a.log2c;
+    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
+    unsigned char* table = smem + cb_bytes;
+    {
+        uint4* dst = reinterpret_cast<uint4*>(table);
+        const int n16 = a.table_bytes / 16;
+        for (int base = 0; base < n16; base += 8 * blockDim.x) {
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = base + u * blockDim.x + threadIdx.x;
+                if (i < n16) v[u] = __ldg(a.table + i);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = base + u * blockDim.x + threadIdx.x;
+                if (i < n16) dst[i] = v[u];
+            }
+        }
+    }
+    const int table_pad = (a.table_bytes + 15) & ~15;
+    unsigned long long* oct_s = reinterpret_cast<unsigned long long*>(table + table_pad) + size_t(warp) * Stage2<NS>::kSlots;
+
+    SearchSmem s;
+    s.cb = smem_addr(smem) + 8u * (threadIdx.x & ((1 << a.log2c) - 1));
+    s.cb_stride = 8u << a.log2c;
+    s.cells = smem_addr(table) - 8u * kMagicBits * uint32_t(a.grid + 1);
+    s.overflow = smem_addr(table + a.off_overflow);
+    s.grid = uint32_t(a.grid);
+    s.K = a.K;
+    s.zlo = pack2(-a.map_zmax, -a.map_zmax);
+    s.c0 = pack2(a.map_c0, a.map_c0);
+    s.c1 = pack2(a.map_c1, a.map_c1);
+    s.c2 = pack2(a.map_c2, a.map_c2);
+    s.bias = pack2(a.map_bias, a.map_bias);
+
+    const int B = a.log2K, B4 = 4 * a.log2K;
+    const unsigned div_magic = 0xffffffffu / unsigned(B4) + 1u;  // ceil(2^32 / (4B))
+    constexpr int kEsz = BF16 ? 2 : 4;
+
+    const int4 span = block_span(a.spans, a.one.d_out);
+    for (int m = span.x; m <= span.z; ++m) {
+        // The warps regroup when the row length changes: nobody may still be inside the previous
+        // matrix (its named barriers and partial sums) when the first warp enters the next one.  The
+        // first pass also waits for the tables.
+        __syncthreads();
+        if (threadIdx.x == 0) cur = a.descs ? a.descs[m] : a.one;
+        __syncthreads();
+        const MatDesc& d = cur;
+        const int d_in = d.d_in, n_pairs = d_in >> 1;
+        const int row_begin = m == span.x ? span.y : 0;
+        const int row_end = m == span.z ? span.w : d.d_out;
+        const int n_seg = (d_in + WE - 1) / WE;
+        const int groups = min(15, n_warps / n_seg);  // named barriers 1..15
+        const int group = warp / n_seg, seg = warp - group * n_seg;
+        const int row0 = row_begin + group;
+        if (group >= groups || row0 >= row_end) continue;
+        const int row_step = groups;
+        const int tg = n_seg * 32;
+        const int oct0 = seg * (WE / 8);
+
+        // per-column constants: t_j = s_j sign_j of the columns the thread loads; reciprocal pair scales
+        // (with the butterfly's sign pattern folded in) of the pairs it holds after the rotation
+        f32x2 t[NS][4];
+        float q[NS][4];
+        bool live[NS];
+        bool risky = false;
+#pragma unroll
+        for (int p = 0; p < NS; ++p) {
+            const int e0 = 8 * (oct0 + Lay::octet_before(lane, p));
+            float cs[8], sgn[8];
+            if (d.chan_scale) {
+                load8f(d.chan_scale, e0, d_in, 1, 1.0f, cs);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) cs[e] = 1.0f;
+            }
+            load8s(d.signs, e0, d_in, 1, sgn);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) t[p][i] = pack2(cs[2 * i] * sgn[2 * i], cs[2 * i + 1] * sgn[2 * i + 1]);
+            const int k0 = 4 * (oct0 + Lay::octet_after(lane, p));
+            live[p] = k0 < n_pairs;
+            load4f(d.sigma, k0, n_pairs, 1, 1.0f, q[p]);
+            const float fl = Lay::negated(lane, p) ? -1.0f : 1.0f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                // q_k = f32(1 / (double)sigma_k): the correctly rounded f32 reciprocal is the same number
+                const float r = live[p] ? __frcp_rn(q[p][i]) : 0.f;
+                // |z| <= q (1 + eps) because |y| <= 1 for a unit row: only a huge reciprocal pair scale can
+                // carry a point beyond the table's reach
+                risky |= !(r < 15000.0f);
+                q[p][i] = fl * r;
+            }
+        }
+        const bool any_risky = __any_sync(kFull, risky);
+
+        const int col0 = seg * WE + 8 * NS * lane;  // first column of this thread
+        const bool have_w = col0 < d_in;            // the fast path needs d_in to be a multiple of 8 NS: all or none
+        const int seg_word0 = 4 * NS * B * seg;     // first packed word of this warp's segment (16 NS B bytes per segment)
+        const bool last_seg = seg == n_seg - 1;
+        double* part_base = &ss_part[0][group * n_seg];
+
+        auto rows = [&](auto mode_tag) {
+            constexpr int MODE = decltype(mode_tag)::value;  // 0 = table, 1 = table with reach check, 2 = exhaustive
+            int parity = 0;
+            for (int row = row0; row < row_end; row += row_step, parity ^= 1) {
+                const char* wp = static_cast<const char*>(cur.W) + ((long long)row * cur.w_row_stride + col0) * kEsz;
+                f32x2 P[NS][4];
+                if (BF16) {
+#pragma unroll
+                    for (int h = 0; h < NS / 2; ++h) {  // two octets (32 bytes) per load
+                        uint32_t w[8];
+                        if (have_w) {
+                            ld_global_256(wp + 32 * h, w);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) w[i] = 0u;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            P[2 * h + (i >> 2)][i & 3] =
+                                mul2(pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u)), t[2 * h + (i >> 2)][i & 3]);
+                    }
+                } else {
+#pragma unroll
+                    for (int p = 0; p < NS; ++p) {
+                        uint32_t w[8];
+                        if (have_w) {
+                            ld_global_256(wp + 32 * p, w);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) w[i] = 0u;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            P[p][i] = mul2(pack2(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1])), t[p][i]);
+                    }
+                }
+                // sum of squares of the row: ss = sum_j (double)x_j^2, per thread, per warp, then per row
+                double* part = part_base + parity * 32;
+                {
+                    double ss = 0.0;
+#pragma unroll
+                    for (int p = 0; p < NS; ++p)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            float x0, x1;
+                            unpack2(P[p][i], x0, x1);
+                            const double d0 = double(x0), d1 = double(x1);
+                            ss = fma(d0, d0, ss);
+                            ss = fma(d1, d1, ss);
+                        }
+                    ss = warp_sum(ss);
+                    if (lane == 0) part[seg] = ss;
+                }
+                // The rotation does not need the norm, so the warps of the row meet only after it.  A
+                // warp can be one row ahead of another at most, hence the two sets of partial sums.
+                fwht2<NS, LOG2B, false>(P, lane);
+                group_barrier(group, tg);
+                float gn = 0.f;
+                if (lane == 0) {  // every warp adds the same numbers in the same order
+                    double total = 0.0;
+                    for (int w = 0; w < n_seg; ++w) total += part[w];
+                    const float r = float(sqrt(total));
+                    // g = f32(c_b / r); 0 for a zero row (all its pairs become the origin) and for a non-finite
+                    // row (its indices are unspecified; the searches accept any input)
+                    if (isfinite(r) && r > 0.f) gn = __fdiv_rn(a.inv_sqrt_b, r);
+                    if (seg == 0) {
+                        cur.row_norm[row] = r;
+                        if (!isfinite(r) && a.status) atomicOr(a.status, 1);
+                    }
+                }
+                gn = __shfl_sync(kFull, gn, 0);
+                const f32x2 gn2 = pack2(gn, gn);
+#pragma unroll
+                for (int p = 0; p < NS; ++p) {
+                    uint32_t v[4];
+                    float2 z[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        float yx, yy;
+                        unpack2(mul2(P[p][i], gn2), yx, yy);
+                        z[i] = make_float2(__fmul_rn(yx, q[p][i]), __fmul_rn(yy, q[p][i]));
+                    }
+                    if (MODE == 0) {
+                        uint2 rec[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) v[i] = uint32_t(search_cell(s, z[i].x, z[i].y, rec[i]));
+                        // rare: one of the four cells has more than four candidates
+                        if (int(cell_overflows(rec[0])) | int(cell_overflows(rec[1])) | int(cell_overflows(rec[2])) | int(cell_overflows(rec[3]))) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                if (cell_overflows(rec[i])) v[i] = uint32_t(search_overflow(s, rec[i], z[i].x, z[i].y));
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            v[i] = uint32_t(MODE == 2 ? search_exhaustive(s, z[i].x, z[i].y) : search_table(s, z[i].x, z[i].y));
+                    }
+                    // two indices fit a 32-bit word (B <= 12); octets beyond the row are staged as zero
+                    unsigned long long packed4 =
+                        (unsigned long long)(v[0] | (v[1] << B)) | ((unsigned long long)(v[2] | (v[3] << B)) << (2 * B));
+                    if (!live[p]) packed4 = 0ull;
+                    oct_s[Stage2<NS>::slot(Lay::octet_after(lane, p))] = packed4;
+                }
+                __syncwarp();
+                // bit packing of the warp's segment: octet o occupies bits [o*4B, (o+1)*4B) (LSB first)
+                const long long pstride = cur.packed_row_stride;
+                uint32_t* out = reinterpret_cast<uint32_t*>(cur.packed + (long long)row * pstride);
+                const int row_words = int(pstride >> 2);
+                const int payload_words = int((((long long)(cur.d_in >> 1) * B + 7) / 8 + 3) / 4);
+                for (int j = lane; j < 4 * NS * B; j += 32) {
+                    const int gw = seg_word0 + j;
+                    if (gw >= payload_words) break;
+                    const unsigned bit0 = unsigned(j) * 32u;
+                    int o = int(__umulhi(bit0, div_magic));  // floor(bit0 / (4B)), octet inside the segment
+                    uint32_t word;
+                    if (B4 >= 32) {
+                        // an octet is at least as wide as a word: bits from octet o and, past its end, from o + 1
+                        const int sh = int(bit0) - o * B4;  // 0 <= sh < 4B
+                        const unsigned long long v0 = oct_s[Stage2<NS>::slot(o)];
+                        const unsigned long long v1 = o + 1 < WE / 8 ? oct_s[Stage2<NS>::slot(o + 1)] : 0ull;
+                        word = uint32_t(v0 >> sh) | uint32_t((v1 << (B4 - sh)) & 0xffffffffull);
+                    } else {
+                        word = 0;
+                        for (; o < WE / 8; ++o) {
+                            const int sh = o * B4 - int(bit0);
+                            if (sh >= 32) break;
+                            const unsigned long long v = oct_s[Stage2<NS>::slot(o)];
+                            word |= sh >= 0 ? uint32_t(v << sh) : uint32_t(v >> (-sh));
+                        }
+                    }
+                    out[gw] = word;
+                }
+                if (last_seg)  // padding up to the row stride is written as zero
+                    for (int gw = payload_words + lane; gw < row_words; gw += 32) out[gw] = 0u;
+                __syncwarp();  // the staging piece is free again
+            }
+        };
+        if (a.brute) rows(std::integral_constant<int, 2>{});
+        else if (any_risky) rows(std::integral_constant<int, 1>{});
+        else rows(std::integral_constant<int, 0>{});
     }
 }
 
@@ -378,7 +693,10 @@ int raise_smem_limit(const void* kernel) {
     std::lock_guard<std::mutex> lock(mu);
     unsigned long long& mask = done[kernel];
     if (mask & bit) return QAMW_OK;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemLimit));
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, kernel);
+    if (e == cudaSuccess)  // the limit covers static and dynamic shared memory together
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemLimit - fa.sharedSizeBytes));
     if (e != cudaSuccess) {
         set_cuda_error("cudaFuncSetAttribute", int(e));
         return QAMW_ERR_NOMEM;
@@ -395,43 +713,81 @@ int launch_decode2(const Decode2Args& a, int blocks, int threads, size_t smem, c
     return launch_check("decode2_kernel");
 }
 
+template <bool BF16, int LOG2B, int NS, int MAXT>
+int launch_encode2(const Encode2Args& a, int blocks, int threads, size_t smem, cudaStream_t st) {
+    int rc = raise_smem_limit(reinterpret_cast<const void*>(&encode2_kernel<BF16, LOG2B, NS, MAXT>));
+    if (rc) return rc;
+    encode2_kernel<BF16, LOG2B, NS, MAXT><<<blocks, threads, smem, st>>>(a);
+    return launch_check("encode2_kernel");
+}
+
+constexpr size_t kEncode2StaticSmem = 512;  // ss_part
+
 }  // namespace
 
 namespace qamw {
 
-int rows_decode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, int block, int K, const float* codebook_dev,
-                uint32_t flags, void* stream) {
+// Contiguous spans of the concatenated row list, one per block, of (nearly) equal cost.  A block works
+// on `groups` rows at a time, each row step taking about the same time whatever the row length, so
+// a row of matrix i costs 1 / groups_i: row_cost[i] = lcm / groups_i in integer units.
+void make_spans(const MatDesc* descs, int n, int n_blocks, const int* row_cost, std::vector<int4>* out) {
+    std::vector<long long> cum(n + 1, 0);
+    for (int i = 0; i < n; ++i) cum[i + 1] = cum[i] + (long long)descs[i].d_out * row_cost[i];
+    const long long total = cum[n];
+    auto locate = [&](long long pos, int* m, int* row) {  // first row that starts at or after cost position `pos`
+        int i = int(std::upper_bound(cum.begin(), cum.end(), pos) - cum.begin()) - 1;
+        i = std::min(std::max(i, 0), n - 1);
+        const long long r = (pos - cum[i] + row_cost[i] - 1) / row_cost[i];
+        *m = i;
+        *row = int(std::min<long long>(r, descs[i].d_out));
+    };
+    out->resize(n_blocks);
+    int m0 = 0, r0 = 0;
+    for (int k = 0; k < n_blocks; ++k) {
+        int m1, r1;
+        if (k == n_blocks - 1) {
+            m1 = n - 1;
+            r1 = descs[n - 1].d_out;
+        } else {
+            locate(total / n_blocks * (k + 1) + (total % n_blocks) * (k + 1) / n_blocks, &m1, &r1);
+        }
+        (*out)[k] = make_int4(m0, r0, m1, r1);
+        m0 = m1;
+        r0 = r1;
+    }
+}
+
+int rows_decode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, const void* spans_dev, int span_blocks,
+                int block, int K, const float* codebook_dev, uint32_t flags, void* stream) {
     constexpr int NS = 4, WE = 256 * NS, kWarps = 16;
     const int log2b = ilog2(block);
     if (log2b < 5 || n <= 0) return QAMW_ERR_SHAPE;
     long long max_rows = 0;
-    int max_seg = 1;
     for (int i = 0; i < n; ++i) {
         const MatDesc& d = descs_host[i];
         if (d.d_in % 16 || d.d_in > WE * kWarps) return QAMW_ERR_SHAPE;
         if (!aligned(d.w_hat, 32) || !aligned(d.packed, 16) || d.packed_row_stride % 16) return QAMW_ERR_SHAPE;
         if (!aligned(d.chan_scale, 16) || !aligned(d.signs, 8) || !aligned(d.sigma, 16)) return QAMW_ERR_SHAPE;
         const int n_seg = (d.d_in + WE - 1) / WE;
-        max_seg = std::max(max_seg, n_seg);
         max_rows = std::max(max_rows, (long long)(d.d_out + kWarps / n_seg - 1) / (kWarps / n_seg));
     }
     if (max_rows == 0) return QAMW_OK;
     Decode2Args a;
     a.descs = descs_dev;
     a.one = descs_host[0];
-    a.n_mats = n;
+    a.spans = static_cast<const int4*>(spans_dev);
     a.codebook = reinterpret_cast<const float2*>(codebook_dev);
     a.K = K;
     a.log2K = ilog2(K);
     a.seg_bytes = 16 * NS * a.log2K;
-    a.stage_bytes = a.seg_bytes + 16;
+    a.stage_bytes = (a.seg_bytes + 16 + 127) & ~127;  // 128-byte aligned ring buffers
     a.inv_sqrt_b = float(1.0 / std::sqrt(double(block)));
     const size_t stage_total = size_t(kWarps) * 2 * a.stage_bytes;
     a.log2c = pick_copies(K, std::min(size_t(128) * 1024, kSmemLimit - stage_total));
     const size_t smem = (size_t(K) * 8 << a.log2c) + stage_total;
     int grid = sm_count();
     if (flags & QAMW_FLAG_HALF_DEVICE) grid = std::max(1, grid / 2);
-    const int blocks = int(std::max<long long>(1, std::min<long long>(grid, max_rows)));
+    const int blocks = spans_dev ? span_blocks : int(std::max<long long>(1, std::min<long long>(grid, max_rows)));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int rc = QAMW_ERR_SHAPE;
     switch (log2b) {
@@ -446,4 +802,288 @@ int rows_decode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, int 
     return rc;
 }
 
+// Warps per block the encoder uses for rows of n_seg segments (0: too long for the fast kernels), and
+// the rows it then has in flight.  22 warps (704 threads, 88 registers each) cover rows up to 11264
+// elements, 28 warps (896 threads, 72 registers) rows up to 14336.
+int encode_warps(int n_seg) { return n_seg <= 22 ? 22 : (n_seg <= 28 ? 28 : 0); }
+int encode_groups(int warps, int n_seg) { return std::min(15, warps / n_seg); }
+int decode_groups(int n_seg) { return 16 / n_seg; }
+constexpr int kCostUnit = 360360;  // divisible by every group count 1..15
+
+int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, const void* spans_dev, int span_blocks,
+                int block, int K, int w_bf16, const ::qamw_codebook* cb, uint32_t flags, int32_t* status, void* stream) {
+    constexpr int NS = 2, WE = 256 * NS;
+    const int log2b = ilog2(block);
+    if (log2b < 5 || log2b > 9 || n <= 0) return QAMW_ERR_SHAPE;
+    const size_t esz = w_bf16 ? 2 : 4;
+    int max_seg = 1;
+    long long rows = 0;
+    for (int i = 0; i < n; ++i) {
+        const MatDesc& d = descs_host[i];
+        if (d.d_in % (8 * NS)) return QAMW_ERR_SHAPE;
+        if (!aligned(d.W, 32) || (size_t(d.w_row_stride) * esz) % 32) return QAMW_ERR_SHAPE;
+        if (!aligned(d.chan_scale, 16) || !aligned(d.signs, 8) || !aligned(d.sigma, 16)) return QAMW_ERR_SHAPE;
+        max_seg = std::max(max_seg, (d.d_in + WE - 1) / WE);
+        rows += d.d_out;
+    }
+    const int warps = encode_warps(max_seg);
+    if (!warps) return QAMW_ERR_SHAPE;
+    if (rows == 0) return QAMW_OK;
+    Encode2Args a;
+    a.descs = descs_dev;
+    a.one = descs_host[0];
+    a.spans = static_cast<const int4*>(spans_dev);
+    a.codebook = static_cast<const float2*>(cb->d_blob);
+    a.table = reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(cb->d_blob) + cb->off_cells);
+    a.table_bytes = int(cb->blob_bytes - cb->off_cells);
+    a.off_overflow = int(cb->off_overflow - cb->off_cells);
+    a.K = K;
+    a.log2K = ilog2(K);
+    a.grid = cb->map.grid;
+    a.map_zmax = cb->map.zmax;
+    a.map_c0 = cb->map.c0;
+    a.map_c1 = cb->map.c1;
+    a.map_c2 = cb->map.c2;
+    a.map_bias = 12582912.0f + float(cb->map.half);
+    a.brute = (flags & QAMW_FLAG_BRUTE_FORCE) ? 1 : 0;
+    a.inv_sqrt_b = float(1.0 / std::sqrt(double(block)));
+    a.status = status;
+    const size_t fixed = ((size_t(a.table_bytes) + 15) & ~size_t(15)) + size_t(warps) * Stage2<NS>::kSlots * 8;
+    if (fixed + size_t(K) * 8 > kSmemLimit - kEncode2StaticSmem) return QAMW_ERR_SHAPE;
+    a.log2c = pick_copies(K, kSmemLimit - kEncode2StaticSmem - fixed);
+    const size_t smem = fixed + (size_t(K) * 8 << a.log2c);
+    int grid = sm_count();
+    if (flags & QAMW_FLAG_HALF_DEVICE) grid = std::max(1, grid / 2);
+    const int blocks = spans_dev ? span_blocks : int(std::max<long long>(1, std::min<long long>(grid, rows)));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int rc = QAMW_ERR_SHAPE;
+#define QAMW_ENC2(LB)                                                                          \
+    case LB:                                                                                   \
+        if (warps == 28)                                                                       \
+            rc = w_bf16 ? launch_encode2<true, LB, NS, 896>(a, blocks, 896, smem, st)          \
+                        : launch_encode2<false, LB, NS, 896>(a, blocks, 896, smem, st);        \
+        else                                                                                   \
+            rc = w_bf16 ? launch_encode2<true, LB, NS, 704>(a, blocks, 704, smem, st)          \
+                        : launch_encode2<false, LB, NS, 704>(a, blocks, 704, smem, st);        \
+        break;
+    switch (log2b) {
+        QAMW_ENC2(5)
+        QAMW_ENC2(6)
+        QAMW_ENC2(7)
+        QAMW_ENC2(8)
+        QAMW_ENC2(9)
+        default: break;
+    }
+#undef QAMW_ENC2
+    return rc;
+}
+
 }  // namespace qamw
+
+// ---------------------------------------------------------------------------------------------
+// batches: all linear weights of a layer or a model behind one handle
+// ---------------------------------------------------------------------------------------------
+// A set of matrices that one launch of a row kernel walks: their descriptors on the device and one
+// span of the concatenated row list per block.
+struct RowSet {
+    std::vector<int> index;         // positions in the batch
+    std::vector<MatDesc> descs;     // host copy of the device array
+    MatDesc* d_descs = nullptr;
+    int4* d_spans = nullptr;
+};
+
+struct qamw_batch {
+    int n = 0;
+    int device = -1;
+    int block = 0, K = 0, w_dtype = 0;
+    const qamw_codebook* cb = nullptr;
+    std::vector<qamw_matrix> items;
+    int n_blocks = 0;
+    RowSet dec;                     // all matrices, spans weighted for the decoder's geometry
+    RowSet enc[2];                  // encoder: rows that fit 22 warps per block, and longer ones (28 warps)
+    std::vector<size_t> ws_offset;  // calibration scratch of item i inside the caller's workspace
+    size_t ws_bytes = 0;
+};
+
+namespace {
+MatDesc make_desc(const qamw_matrix& it) {
+    MatDesc d{};
+    d.W = it.W;
+    d.chan_scale = it.chan_scale;
+    d.signs = it.signs;
+    d.sigma = it.sigma;
+    d.act_rms = it.act_rms;
+    d.packed = it.packed;
+    d.row_norm = it.row_norm;
+    d.w_hat = it.w_hat_bf16;
+    d.dist4 = it.dist4;
+    d.w_row_stride = it.p.w_row_stride;
+    d.packed_row_stride = it.p.packed_row_stride;
+    d.d_out = it.p.d_out;
+    d.d_in = it.p.d_in;
+    return d;
+}
+}  // namespace
+
+namespace {
+void free_row_set(RowSet& r) {
+    if (r.d_descs) cudaFree(r.d_descs);
+    if (r.d_spans) cudaFree(r.d_spans);
+    r.d_descs = nullptr;
+    r.d_spans = nullptr;
+}
+cudaError_t upload_row_set(RowSet& r, int n_blocks, const std::vector<int>& row_cost) {
+    if (r.descs.empty()) return cudaSuccess;
+    std::vector<int4> spans;
+    make_spans(r.descs.data(), int(r.descs.size()), n_blocks, row_cost.data(), &spans);
+    cudaError_t e = cudaMalloc(&r.d_descs, sizeof(MatDesc) * r.descs.size());
+    if (e == cudaSuccess) e = cudaMemcpy(r.d_descs, r.descs.data(), sizeof(MatDesc) * r.descs.size(), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMalloc(&r.d_spans, sizeof(int4) * spans.size());
+    if (e == cudaSuccess) e = cudaMemcpy(r.d_spans, spans.data(), sizeof(int4) * spans.size(), cudaMemcpyHostToDevice);
+    return e;
+}
+}  // namespace
+
+extern "C" int qamw_batch_create(const qamw_matrix* items, int n, const qamw_codebook* cb, qamw_batch** out) {
+    if (!items || n <= 0 || !cb || !out) return QAMW_ERR_ARG;
+    *out = nullptr;
+    for (int i = 0; i < n; ++i) {
+        int rc = check_matrix_params(&items[i].p);
+        if (rc) return rc;
+        const qamw_params& p = items[i].p;
+        if (p.block != items[0].p.block || p.K != items[0].p.K || p.w_dtype != items[0].p.w_dtype) return QAMW_ERR_ARG;
+        if (p.K != cb->K || !items[i].signs) return QAMW_ERR_ARG;
+        const size_t row_bytes = qamw_packed_row_bytes(p.d_in, p.K);
+        if (p.packed_row_stride < (long long)row_bytes || p.packed_row_stride % 4) return QAMW_ERR_ALIGN;
+        if (reinterpret_cast<uintptr_t>(items[i].packed) % 4) return QAMW_ERR_ALIGN;
+    }
+    int device = -1;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) {
+        set_cuda_error("qamw_batch_create", int(e));
+        return QAMW_ERR_CUDA;
+    }
+    if (device != cb->device) return QAMW_ERR_ARG;  // the codebook lives on another device
+    qamw_batch* b = new (std::nothrow) qamw_batch();
+    if (!b) return QAMW_ERR_NOMEM;
+    b->n = n;
+    b->device = device;
+    b->block = items[0].p.block;
+    b->K = items[0].p.K;
+    b->w_dtype = items[0].p.w_dtype;
+    b->cb = cb;
+    b->items.assign(items, items + n);
+    b->n_blocks = sm_count();
+    std::vector<int> dec_cost, enc_cost[2];
+    for (int i = 0; i < n; ++i) {
+        const MatDesc d = make_desc(items[i]);
+        b->ws_offset.push_back(b->ws_bytes);
+        b->ws_bytes += (qamw_calibrate_workspace_bytes(&items[i].p) + 255) & ~size_t(255);
+        const int seg4 = (d.d_in + 1023) / 1024, seg2 = (d.d_in + 511) / 512;
+        b->dec.index.push_back(i);
+        b->dec.descs.push_back(d);
+        dec_cost.push_back(kCostUnit / std::max(1, decode_groups(std::min(seg4, 16))));
+        const int warps = encode_warps(seg2);
+        const int c = warps == 22 ? 0 : 1;  // rows too long for either class end up in class 1 and fall back later
+        b->enc[c].index.push_back(i);
+        b->enc[c].descs.push_back(d);
+        enc_cost[c].push_back(kCostUnit / std::max(1, encode_groups(warps ? warps : 28, std::min(seg2, 28))));
+    }
+    e = upload_row_set(b->dec, b->n_blocks, dec_cost);
+    for (int c = 0; c < 2 && e == cudaSuccess; ++c) e = upload_row_set(b->enc[c], b->n_blocks, enc_cost[c]);
+    if (e != cudaSuccess) {
+        set_cuda_error("qamw_batch_create", int(e));
+        qamw_batch_destroy(b);
+        return QAMW_ERR_CUDA;
+    }
+    *out = b;
+    return QAMW_OK;
+}
+
+extern "C" void qamw_batch_destroy(qamw_batch* b) {
+    if (!b) return;
+    free_row_set(b->dec);
+    free_row_set(b->enc[0]);
+    free_row_set(b->enc[1]);
+    delete b;
+}
+
+extern "C" size_t qamw_batch_workspace_bytes(const qamw_batch* b) { return b ? b->ws_bytes : 0; }
+
+extern "C" int qamw_calibrate_batch(const qamw_batch* b, void* workspace, size_t workspace_bytes, int32_t* status_out,
+                                    void* stream) {
+    if (!b || !workspace) return QAMW_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % 8) return QAMW_ERR_ALIGN;
+    if (workspace_bytes < b->ws_bytes) return QAMW_ERR_NOMEM;
+    for (int i = 0; i < b->n; ++i)
+        if (!b->items[i].W || !b->items[i].sigma) return QAMW_ERR_ARG;
+    for (int i = 0; i < b->n; ++i) {
+        const qamw_matrix& it = b->items[i];
+        int rc = qamw_calibrate(it.W, &it.p, it.chan_scale, it.signs, it.sigma,
+                                static_cast<unsigned char*>(workspace) + b->ws_offset[i],
+                                workspace_bytes - b->ws_offset[i], status_out, stream);
+        if (rc) return rc;
+    }
+    return QAMW_OK;
+}
+
+extern "C" int qamw_encode_batch(const qamw_batch* b, int32_t* status_out, void* stream) {
+    if (!b) return QAMW_ERR_ARG;
+    for (int i = 0; i < b->n; ++i) {
+        const qamw_matrix& it = b->items[i];
+        if (!it.W || !it.sigma || !it.packed || !it.row_norm) return QAMW_ERR_ARG;
+    }
+    const uint32_t flags = b->items[0].p.flags;
+    for (int c = 0; c < 2; ++c) {  // one launch per class of row lengths
+        const RowSet& set = b->enc[c];
+        if (set.descs.empty()) continue;
+        int rc = QAMW_ERR_SHAPE;
+        if (!(flags & QAMW_FLAG_GENERAL_KERNELS))
+            rc = rows_encode(set.d_descs, set.descs.data(), int(set.descs.size()), set.d_spans, b->n_blocks, b->block, b->K,
+                             b->w_dtype == QAMW_DTYPE_BF16, b->cb, flags, status_out, stream);
+        if (rc == QAMW_ERR_SHAPE) {  // some matrix of the class needs the general kernel: one call per matrix
+            rc = QAMW_OK;
+            for (size_t k = 0; k < set.index.size() && rc == QAMW_OK; ++k) {
+                const qamw_matrix& it = b->items[set.index[k]];
+                rc = qamw_encode(it.W, &it.p, it.chan_scale, it.signs, it.sigma, b->cb, it.packed, it.row_norm, status_out,
+                                 stream);
+            }
+        }
+        if (rc) return rc;
+    }
+    return QAMW_OK;
+}
+
+extern "C" int qamw_decode_batch(const qamw_batch* b, void* stream) {
+    if (!b) return QAMW_ERR_ARG;
+    for (int i = 0; i < b->n; ++i) {
+        const qamw_matrix& it = b->items[i];
+        if (!it.sigma || !it.packed || !it.row_norm || !it.w_hat_bf16) return QAMW_ERR_ARG;
+    }
+    const uint32_t flags = b->items[0].p.flags;
+    int rc = QAMW_ERR_SHAPE;
+    if (!(flags & QAMW_FLAG_GENERAL_KERNELS))
+        rc = rows_decode(b->dec.d_descs, b->dec.descs.data(), b->n, b->dec.d_spans, b->n_blocks, b->block, b->K,
+                         static_cast<const float*>(b->cb->d_blob), flags, stream);
+    if (rc != QAMW_ERR_SHAPE) return rc;
+    for (int i = 0; i < b->n; ++i) {  // some matrix needs the general kernel: one call per matrix
+        const qamw_matrix& it = b->items[i];
+        rc = qamw_decode(it.packed, it.row_norm, it.chan_scale, it.signs, it.sigma, b->cb, &it.p, it.w_hat_bf16, stream);
+        if (rc) return rc;
+    }
+    return QAMW_OK;
+}
+
+extern "C" int qamw_distortion_batch(const qamw_batch* b, void* stream) {
+    if (!b) return QAMW_ERR_ARG;
+    for (int i = 0; i < b->n; ++i) {
+        const qamw_matrix& it = b->items[i];
+        if (!it.W || !it.w_hat_bf16 || !it.dist4) return QAMW_ERR_ARG;
+    }
+    for (int i = 0; i < b->n; ++i) {
+        const qamw_matrix& it = b->items[i];
+        int rc = qamw_distortion(it.W, it.w_hat_bf16, it.act_rms, &it.p, it.dist4, stream);
+        if (rc) return rc;
+    }
+    return QAMW_OK;
+}
