@@ -1,6 +1,8 @@
 """Whole-model driver over the C ABI: calibrate -> encode -> decode -> distortion for every
 linear weight of a (synthetic) checkpoint.  This is the call a user of the library makes to
-quantise a model; each phase is a plain loop of library calls, one per weight matrix.
+quantise a model.  Encode and decode go through one qamw_batch (a persistent launch per phase
+that walks all matrices); calibration and distortion are one library call per matrix, dealt
+onto a few side streams.
 """
 from __future__ import annotations
 
@@ -64,6 +66,8 @@ class ModelCodec:
     slots: List[MatrixSlot] = field(default_factory=list)
     workspace: Optional[torch.Tensor] = None
     status: Optional[torch.Tensor] = None
+    batch: Optional[q.Batch] = None
+    use_batch: bool = True
     _meta_cache: Dict[int, Tuple[torch.Tensor, torch.Tensor]] = field(default_factory=dict)
 
     @classmethod
@@ -81,7 +85,15 @@ class ModelCodec:
                 ws_bytes = max(ws_bytes, q.calibrate_workspace_bytes(mc.slots[-1].params))
             mc.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
             mc.status = torch.zeros(1, dtype=torch.int32, device=dev)
+            mc.finalize()
         return mc
+
+    def finalize(self):
+        """Build the batch handle over all matrices added so far (call again after add_matrix)."""
+        with torch.cuda.device(self.device):
+            mats = [q.make_matrix(s.params, s.W, s.chan_scale, s.signs, s.sigma, s.act_rms, s.packed, s.row_norm,
+                                  s.w_hat, s.dist) for s in self.slots]
+            self.batch = q.Batch(mats, self.codebook) if mats else None
 
     def add_matrix(self, name: str, W: torch.Tensor, act_rms: torch.Tensor, sign_seed: int = q.DEFAULT_SIGN_SEED):
         spec, dev = self.spec, self.device
@@ -134,10 +146,14 @@ class ModelCodec:
         self._phase(lambda s, ws, st: q.calibrate(s.W, s.params, s.chan_scale, s.signs, s.sigma, ws, self.status, st))
 
     def encode_all(self):
+        if self.use_batch and self.batch is not None:
+            return self.batch.encode(self.status)
         self._phase(lambda s, ws, st: q.encode(s.W, s.params, s.chan_scale, s.signs, s.sigma, self.codebook, s.packed,
                                                s.row_norm, self.status, st))
 
     def decode_all(self):
+        if self.use_batch and self.batch is not None:
+            return self.batch.decode()
         self._phase(lambda s, ws, st: q.decode(s.packed, s.row_norm, s.chan_scale, s.signs, s.sigma, self.codebook,
                                                s.params, s.w_hat, st))
 
@@ -167,8 +183,14 @@ class ModelCodec:
         return enc, dec
 
     def kernel_launches_per_step(self) -> int:
-        # calibrate = 2 kernels, encode 1, decode 1, distortion 1 (its memset is not a kernel of ours)
-        return 5 * len(self.slots)
+        # per matrix: calibrate = 2 kernels, distortion 1 (its memset is not a kernel of ours); encode and
+        # decode are per matrix too unless batched: then one decode launch and one encode launch per
+        # class of row lengths (rows of up to 11264 elements, longer rows)
+        n = len(self.slots)
+        if self.use_batch and self.batch is not None:
+            enc = len({s.d_in > 11264 for s in self.slots})
+            return 3 * n + enc + 1
+        return 5 * n
 
     def totals(self, group=None) -> Dict[str, float]:
         """Error figures over all matrices of all ranks (see combine_distortion)."""
