@@ -175,6 +175,19 @@ def test_argument_errors_are_reported_before_any_launch():
     assert lib.qamw_calibrate(ptr, C.byref(params()), None, ptr, ptr, None, 0, None, None) == q.ERR_ARG
     assert lib.qamw_calibrate_static(ptr, C.byref(params(block=96)), None, ptr, ptr, None, None) == q.ERR_SHAPE
     assert lib.qamw_rotate(ptr, None, None, ptr, ptr, ptr, None, None) == q.ERR_ARG
+    # batches: argument checks come before any CUDA call
+    hb = C.c_void_p()
+    item = q.Matrix(params(block=96), ptr.value, None, ptr.value, ptr.value, None, ptr.value, ptr.value, ptr.value, ptr.value)
+    arr = (q.Matrix * 1)(item)
+    assert lib.qamw_batch_create(None, 1, ptr, C.byref(hb)) == q.ERR_ARG
+    assert lib.qamw_batch_create(arr, 0, ptr, C.byref(hb)) == q.ERR_ARG
+    assert lib.qamw_batch_create(arr, 1, None, C.byref(hb)) == q.ERR_ARG
+    assert lib.qamw_batch_create(arr, 1, ptr, C.byref(hb)) == q.ERR_SHAPE  # block is not a power of two
+    assert lib.qamw_encode_batch(None, None, None) == q.ERR_ARG
+    assert lib.qamw_decode_batch(None, None) == q.ERR_ARG
+    assert lib.qamw_distortion_batch(None, None) == q.ERR_ARG
+    assert lib.qamw_calibrate_batch(None, ptr, 64, None, None) == q.ERR_ARG
+    assert lib.qamw_batch_workspace_bytes(None) == 0
     h = C.c_void_p()
     cbk = np.zeros((4, 2), np.float32)
     assert lib.qamw_codebook_create(cbk.ctypes.data, 3, 0, C.byref(h)) == q.ERR_SHAPE
