@@ -523,39 +523,36 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
         auto rows = [&](auto mode_tag) {
             constexpr int MODE = decltype(mode_tag)::value;  // 0 = table, 1 = table with reach check, 2 = exhaustive
             int parity = 0;
-            for (int row = row0; row < row_end; row += row_step, parity ^= 1) {
+            // raw bits of the thread's elements of one row; the next row is fetched as soon as this one
+            // has been converted, so its latency hides behind the rotation and the search
+            constexpr int kRaw = BF16 ? 4 * NS : 8 * NS;
+            uint32_t raw[kRaw];
+            auto fetch = [&](int row) {
                 const char* wp = static_cast<const char*>(cur.W) + ((long long)row * cur.w_row_stride + col0) * kEsz;
+#pragma unroll
+                for (int h = 0; h < kRaw / 8; ++h) {
+                    uint32_t w[8];
+                    ld_global_256(wp + 32 * h, w);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) raw[8 * h + i] = w[i];
+                }
+            };
+#pragma unroll
+            for (int i = 0; i < kRaw; ++i) raw[i] = 0u;
+            if (have_w) fetch(row0);
+            for (int row = row0; row < row_end; row += row_step, parity ^= 1) {
                 f32x2 P[NS][4];
                 if (BF16) {
 #pragma unroll
-                    for (int h = 0; h < NS / 2; ++h) {  // two octets (32 bytes) per load
-                        uint32_t w[8];
-                        if (have_w) {
-                            ld_global_256(wp + 32 * h, w);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) w[i] = 0u;
-                        }
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            P[2 * h + (i >> 2)][i & 3] =
-                                mul2(pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u)), t[2 * h + (i >> 2)][i & 3]);
-                    }
+                    for (int i = 0; i < 4 * NS; ++i)
+                        P[i >> 2][i & 3] = mul2(pack2(__uint_as_float(raw[i] << 16), __uint_as_float(raw[i] & 0xffff0000u)),
+                                                t[i >> 2][i & 3]);
                 } else {
 #pragma unroll
-                    for (int p = 0; p < NS; ++p) {
-                        uint32_t w[8];
-                        if (have_w) {
-                            ld_global_256(wp + 32 * p, w);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) w[i] = 0u;
-                        }
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            P[p][i] = mul2(pack2(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1])), t[p][i]);
-                    }
+                    for (int i = 0; i < 4 * NS; ++i)
+                        P[i >> 2][i & 3] = mul2(pack2(__uint_as_float(raw[2 * i]), __uint_as_float(raw[2 * i + 1])), t[i >> 2][i & 3]);
                 }
+                if (have_w && row + row_step < row_end) fetch(row + row_step);
                 // sum of squares of the row: ss = sum_j (double)x_j^2, per thread, per warp, then per row
                 double* part = part_base + parity * 32;
                 {
@@ -802,11 +799,22 @@ int rows_decode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, cons
     return rc;
 }
 
-// Warps per block the encoder uses for rows of n_seg segments (0: too long for the fast kernels), and
-// the rows it then has in flight.  22 warps (704 threads, 88 registers each) cover rows up to 11264
-// elements, 28 warps (896 threads, 72 registers) rows up to 14336.
-int encode_warps(int n_seg) { return n_seg <= 22 ? 22 : (n_seg <= 28 ? 28 : 0); }
+// Block sizes of the encoder: 20, 24 or 28 warps.  The register file is split over the four
+// schedulers of an SM, 16384 registers each, so 5, 6 or 7 warps per scheduler leave 96, 80 or 72
+// registers per thread.  A row of n_seg segments takes the size that keeps most warps busy (whole
+// groups of n_seg warps, at most 15 groups), and among equals the smallest: 0 if the row is too long.
 int encode_groups(int warps, int n_seg) { return std::min(15, warps / n_seg); }
+int encode_warps(int n_seg) {
+    int best = 0, best_busy = 0;
+    for (int w = 20; w <= 28; w += 4) {
+        const int busy = encode_groups(w, n_seg) * n_seg;
+        if (busy > best_busy) {
+            best = w;
+            best_busy = busy;
+        }
+    }
+    return best;
+}
 int decode_groups(int n_seg) { return 16 / n_seg; }
 constexpr int kCostUnit = 360360;  // divisible by every group count 1..15
 
@@ -816,18 +824,19 @@ int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, cons
     const int log2b = ilog2(block);
     if (log2b < 5 || log2b > 9 || n <= 0) return QAMW_ERR_SHAPE;
     const size_t esz = w_bf16 ? 2 : 4;
-    int max_seg = 1;
+    int max_seg = 1, warps = 0;
     long long rows = 0;
     for (int i = 0; i < n; ++i) {
         const MatDesc& d = descs_host[i];
         if (d.d_in % (8 * NS)) return QAMW_ERR_SHAPE;
         if (!aligned(d.W, 32) || (size_t(d.w_row_stride) * esz) % 32) return QAMW_ERR_SHAPE;
         if (!aligned(d.chan_scale, 16) || !aligned(d.signs, 8) || !aligned(d.sigma, 16)) return QAMW_ERR_SHAPE;
-        max_seg = std::max(max_seg, (d.d_in + WE - 1) / WE);
+        const int n_seg = (d.d_in + WE - 1) / WE;
+        max_seg = std::max(max_seg, n_seg);
+        warps = std::max(warps, encode_warps(n_seg));
         rows += d.d_out;
     }
-    const int warps = encode_warps(max_seg);
-    if (!warps) return QAMW_ERR_SHAPE;
+    if (max_seg > warps) return QAMW_ERR_SHAPE;  // also: a row too long for any block size
     if (rows == 0) return QAMW_OK;
     Encode2Args a;
     a.descs = descs_dev;
@@ -862,9 +871,12 @@ int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, cons
         if (warps == 28)                                                                       \
             rc = w_bf16 ? launch_encode2<true, LB, NS, 896>(a, blocks, 896, smem, st)          \
                         : launch_encode2<false, LB, NS, 896>(a, blocks, 896, smem, st);        \
+        else if (warps == 24)                                                                  \
+            rc = w_bf16 ? launch_encode2<true, LB, NS, 768>(a, blocks, 768, smem, st)          \
+                        : launch_encode2<false, LB, NS, 768>(a, blocks, 768, smem, st);        \
         else                                                                                   \
-            rc = w_bf16 ? launch_encode2<true, LB, NS, 704>(a, blocks, 704, smem, st)          \
-                        : launch_encode2<false, LB, NS, 704>(a, blocks, 704, smem, st);        \
+            rc = w_bf16 ? launch_encode2<true, LB, NS, 640>(a, blocks, 640, smem, st)          \
+                        : launch_encode2<false, LB, NS, 640>(a, blocks, 640, smem, st);        \
         break;
     switch (log2b) {
         QAMW_ENC2(5)
@@ -900,7 +912,7 @@ struct qamw_batch {
     std::vector<qamw_matrix> items;
     int n_blocks = 0;
     RowSet dec;                     // all matrices, spans weighted for the decoder's geometry
-    RowSet enc[2];                  // encoder: rows that fit 22 warps per block, and longer ones (28 warps)
+    RowSet enc[3];                  // encoder: one set per block size (20, 24, 28 warps)
     std::vector<size_t> ws_offset;  // calibration scratch of item i inside the caller's workspace
     size_t ws_bytes = 0;
 };
@@ -974,7 +986,7 @@ extern "C" int qamw_batch_create(const qamw_matrix* items, int n, const qamw_cod
     b->cb = cb;
     b->items.assign(items, items + n);
     b->n_blocks = sm_count();
-    std::vector<int> dec_cost, enc_cost[2];
+    std::vector<int> dec_cost, enc_cost[3];
     for (int i = 0; i < n; ++i) {
         const MatDesc d = make_desc(items[i]);
         b->ws_offset.push_back(b->ws_bytes);
@@ -984,13 +996,13 @@ extern "C" int qamw_batch_create(const qamw_matrix* items, int n, const qamw_cod
         b->dec.descs.push_back(d);
         dec_cost.push_back(kCostUnit / std::max(1, decode_groups(std::min(seg4, 16))));
         const int warps = encode_warps(seg2);
-        const int c = warps == 22 ? 0 : 1;  // rows too long for either class end up in class 1 and fall back later
+        const int c = warps == 20 ? 0 : (warps == 24 ? 1 : 2);  // rows too long for any size end up in the last set and fall back later
         b->enc[c].index.push_back(i);
         b->enc[c].descs.push_back(d);
         enc_cost[c].push_back(kCostUnit / std::max(1, encode_groups(warps ? warps : 28, std::min(seg2, 28))));
     }
     e = upload_row_set(b->dec, b->n_blocks, dec_cost);
-    for (int c = 0; c < 2 && e == cudaSuccess; ++c) e = upload_row_set(b->enc[c], b->n_blocks, enc_cost[c]);
+    for (int c = 0; c < 3 && e == cudaSuccess; ++c) e = upload_row_set(b->enc[c], b->n_blocks, enc_cost[c]);
     if (e != cudaSuccess) {
         set_cuda_error("qamw_batch_create", int(e));
         qamw_batch_destroy(b);
@@ -1003,8 +1015,7 @@ extern "C" int qamw_batch_create(const qamw_matrix* items, int n, const qamw_cod
 extern "C" void qamw_batch_destroy(qamw_batch* b) {
     if (!b) return;
     free_row_set(b->dec);
-    free_row_set(b->enc[0]);
-    free_row_set(b->enc[1]);
+    for (int c = 0; c < 3; ++c) free_row_set(b->enc[c]);
     delete b;
 }
 
@@ -1034,7 +1045,7 @@ extern "C" int qamw_encode_batch(const qamw_batch* b, int32_t* status_out, void*
         if (!it.W || !it.sigma || !it.packed || !it.row_norm) return QAMW_ERR_ARG;
     }
     const uint32_t flags = b->items[0].p.flags;
-    for (int c = 0; c < 2; ++c) {  // one launch per class of row lengths
+    for (int c = 0; c < 3; ++c) {  // one launch per block size
         const RowSet& set = b->enc[c];
         if (set.descs.empty()) continue;
         int rc = QAMW_ERR_SHAPE;
