@@ -305,3 +305,67 @@ def train_codebook(K, n_samples=1 << 20, seed=0, max_iters=100, rel_tol=1e-6, wa
 def codebook_mse(codebook, n_samples, seed) -> float:
     cb = _c(codebook, np.float32)
     return float(lib().orc_codebook_mse(_p(cb), C.c_int(cb.shape[0]), C.c_uint64(n_samples), C.c_uint64(seed)))
+
+
+# ------------------------------------------------------------------------------- polar baseline
+def rayleigh_lloyd_max(n_levels: int, max_iters: int = 5000):
+    """N-level Lloyd-Max quantiser of the unit Rayleigh density -> (f32 levels, C_LM of those levels)."""
+    levels = np.empty(n_levels, np.float32)
+    L = lib()
+    L.orc_rayleigh_lloyd_max.restype = C.c_double
+    c_lm = L.orc_rayleigh_lloyd_max(C.c_int(n_levels), C.c_int(max_iters), _p(levels))
+    return levels, float(c_lm)
+
+
+def rayleigh_distortion(levels) -> float:
+    lv = _c(levels, np.float64)
+    L = lib()
+    L.orc_rayleigh_distortion.restype = C.c_double
+    return float(L.orc_rayleigh_distortion(_p(lv), C.c_int(lv.shape[0])))
+
+
+def polar_codebook(levels, Ba: int, Bp: int) -> np.ndarray:
+    lv = _c(levels, np.float32)
+    out = np.empty((1 << (Ba + Bp), 2), np.float32)
+    lib().orc_polar_codebook(_p(lv), C.c_int(Ba), C.c_int(Bp), _p(out))
+    return out
+
+
+def polar_quantize(z, levels, Ba: int, Bp: int):
+    """Polar quantiser for each point of z[n,2] -> (idx, amplitude margin, phase margin)."""
+    z = _c(z, np.float64).reshape(-1, 2)
+    lv = _c(levels, np.float32)
+    idx = np.empty(z.shape[0], np.int32)
+    ma = np.empty(z.shape[0], np.float64)
+    mp = np.empty(z.shape[0], np.float64)
+    L = lib()
+    L.orc_polar_quantize.restype = C.c_int
+    a, b = C.c_double(), C.c_double()
+    for i in range(z.shape[0]):
+        idx[i] = L.orc_polar_quantize(C.c_double(z[i, 0]), C.c_double(z[i, 1]), _p(lv), C.c_int(Ba), C.c_int(Bp),
+                                      C.byref(a), C.byref(b))
+        ma[i], mp[i] = a.value, b.value
+    return idx, ma, mp
+
+
+def encode_polar(W, b, levels, Ba, Bp, chan_scale, signs, sigma, packed_row_stride=None, diagnostics=False):
+    """Encoder with the polar quantiser (Section 3.5) instead of the 2-D search."""
+    W = np.ascontiguousarray(W)
+    d_out, d_in = W.shape
+    lv = _c(levels, np.float32)
+    K = 1 << (Ba + Bp)
+    rb = packed_row_bytes(d_in, K)
+    stride = rb if packed_row_stride is None else int(packed_row_stride)
+    packed = np.zeros((d_out, stride), np.uint8)
+    norms = np.empty(d_out, np.float32)
+    z = idx = ma = mp = None
+    if diagnostics:
+        z = np.empty((d_out, d_in // 2, 2), np.float32)
+        idx = np.empty((d_out, d_in // 2), np.int32)
+        ma = np.empty((d_out, d_in // 2), np.float64)
+        mp = np.empty((d_out, d_in // 2), np.float64)
+    rc = lib().orc_encode_polar(_p(W), C.c_int(_w_dtype(W)), C.c_int(d_out), C.c_int(d_in), C.c_int64(d_in),
+                                C.c_int(b), C.c_int(Ba), C.c_int(Bp), _p(_c(chan_scale, np.float32)),
+                                _p(_c(signs, np.int8)), _p(_c(sigma, np.float32)), _p(lv), _p(packed), C.c_int64(stride),
+                                _p(norms), _p(z), _p(idx), _p(ma), _p(mp))
+    return dict(status=int(rc), packed=packed, row_norm=norms, z=z, idx=idx, margin_a=ma, margin_p=mp)

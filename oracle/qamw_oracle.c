@@ -667,3 +667,184 @@ double orc_codebook_mse(const float *codebook, int K, uint64_t n, uint64_t seed)
     free(cb);
     return D;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Polar baseline (Section 3.5; Corollary "Rayleigh-Lloyd polar distortion     */
+/* bound" and the Remark after it).                                           */
+/* ------------------------------------------------------------------------- */
+
+/* Composite Simpson rule for the three moments of the unit Rayleigh density
+ * f(r) = r exp(-r^2/2) on [a, b]: m[q] = int r^q f(r) dr, q = 0, 1, 2. */
+static void rayleigh_moments(double a, double b, int n_sub, double m[3]) {
+    m[0] = m[1] = m[2] = 0.0;
+    if (!(b > a)) return;
+    if (n_sub % 2) ++n_sub;
+    double h = (b - a) / n_sub;
+    for (int i = 0; i <= n_sub; ++i) {
+        double r = a + h * i;
+        double w = (i == 0 || i == n_sub) ? 1.0 : ((i % 2) ? 4.0 : 2.0);
+        double f = r * exp(-0.5 * r * r) * w;
+        m[0] += f;
+        m[1] += f * r;
+        m[2] += f * r * r;
+    }
+    m[0] *= h / 3.0;
+    m[1] *= h / 3.0;
+    m[2] *= h / 3.0;
+}
+
+#define ORC_RAYLEIGH_RMAX 8.0 /* integration cut-off named in the Remark */
+
+/* Distortion int_0^Rmax (r - Q(r))^2 f(r) dr of the nearest-level quantiser with
+ * the given levels (ascending), cells bounded by the midpoints. */
+double orc_rayleigh_distortion(const double *levels, int n) {
+    double D = 0.0;
+    for (int j = 0; j < n; ++j) {
+        double lo = j == 0 ? 0.0 : 0.5 * (levels[j - 1] + levels[j]);
+        double hi = j == n - 1 ? ORC_RAYLEIGH_RMAX : 0.5 * (levels[j] + levels[j + 1]);
+        double m[3];
+        rayleigh_moments(lo, hi, 4096, m);
+        D += m[2] - 2.0 * levels[j] * m[1] + levels[j] * levels[j] * m[0];
+    }
+    return D;
+}
+
+/* N-level Lloyd-Max quantiser of the unit Rayleigh density under squared error:
+ * start from the quantiles r_j = sqrt(-2 ln(1 - (j + 1/2)/N)), then alternate
+ * "cell boundaries = midpoints of the levels" and "level = centroid of its cell"
+ * (numerically integrated on [0, 8]) until no level moves by more than 1e-13 or
+ * max_iters rounds.  levels_out: f32 (the practical codebook); returns the
+ * numerically integrated distortion C_LM of those f32 levels. */
+double orc_rayleigh_lloyd_max(int n, int max_iters, float *levels_out) {
+    double *l = (double *)malloc(sizeof(double) * (size_t)n);
+    for (int j = 0; j < n; ++j) l[j] = sqrt(-2.0 * log(1.0 - ((double)j + 0.5) / (double)n));
+    for (int it = 0; it < max_iters; ++it) {
+        double move = 0.0, prev_level = 0.0, next;
+        for (int j = 0; j < n; ++j) {
+            double lo = j == 0 ? 0.0 : 0.5 * (prev_level + l[j]);
+            double hi = j == n - 1 ? ORC_RAYLEIGH_RMAX : 0.5 * (l[j] + l[j + 1]);
+            double m[3];
+            rayleigh_moments(lo, hi, 4096, m);
+            next = m[0] > 0.0 ? m[1] / m[0] : l[j];
+            prev_level = l[j]; /* boundaries of this round use the levels of the previous round */
+            if (fabs(next - l[j]) > move) move = fabs(next - l[j]);
+            l[j] = next;
+        }
+        if (move < 1e-13) break;
+    }
+    for (int j = 0; j < n; ++j) {
+        levels_out[j] = (float)l[j];
+        l[j] = (double)levels_out[j];
+    }
+    double D = orc_rayleigh_distortion(l, n);
+    free(l);
+    return D;
+}
+
+/* The K = 2^(Ba+Bp) reconstruction points of the polar codec as one table:
+ * index = (p << Ba) | a, point = level_a (cos phi_p, sin phi_p) with the bin
+ * centres phi_p = (2p + 1) pi / N_p of the Corollary, rounded to f32. */
+void orc_polar_codebook(const float *levels, int Ba, int Bp, float *codebook_out) {
+    const double pi = 3.14159265358979323846264338327950288;
+    int Na = 1 << Ba, Np = 1 << Bp;
+    for (int p = 0; p < Np; ++p) {
+        double phi = (2.0 * p + 1.0) * pi / (double)Np;
+        for (int a = 0; a < Na; ++a) {
+            int idx = (p << Ba) | a;
+            codebook_out[2 * idx] = (float)((double)levels[a] * cos(phi));
+            codebook_out[2 * idx + 1] = (float)((double)levels[a] * sin(phi));
+        }
+    }
+}
+
+/* Polar quantiser of one point: amplitude to the nearest level (lowest index on
+ * ties), phase theta in [0, 2 pi) to the bin floor(theta / (2 pi / N_p)); the
+ * origin goes to bin 0.  margin_a: (gap between the distances to the two
+ * nearest levels) / amplitude; margin_p: distance in radians to the nearest
+ * bin boundary (pi when there is one bin or the point is the origin). */
+int orc_polar_quantize(double zx, double zy, const float *levels, int Ba, int Bp, double *margin_a,
+                       double *margin_p) {
+    const double pi = 3.14159265358979323846264338327950288;
+    int Na = 1 << Ba, Np = 1 << Bp;
+    double r = sqrt(zx * zx + zy * zy);
+    int a = 0;
+    double d1 = INFINITY, d2 = INFINITY;
+    for (int j = 0; j < Na; ++j) {
+        double d = fabs(r - (double)levels[j]);
+        if (d < d1) {
+            d2 = d1;
+            d1 = d;
+            a = j;
+        } else if (d < d2) {
+            d2 = d;
+        }
+    }
+    if (margin_a) *margin_a = Na > 1 ? (d2 - d1) / (r > 1e-300 ? r : 1e-300) : INFINITY;
+    int p = 0;
+    double mp = pi;
+    if (Np > 1 && !(zx == 0.0 && zy == 0.0)) {
+        double theta = atan2(zy, zx);
+        if (theta < 0.0) theta += 2.0 * pi;
+        double width = 2.0 * pi / (double)Np;
+        p = (int)floor(theta / width);
+        if (p >= Np) p = Np - 1;
+        double lo = theta - width * p, hi = width * (p + 1) - theta;
+        mp = lo < hi ? lo : hi;
+    }
+    if (margin_p) *margin_p = mp;
+    return (p << Ba) | a;
+}
+
+/* Encoder with the polar quantiser in place of the nearest-codeword search:
+ * everything up to z_k as in orc_encode, then idx_k = orc_polar_quantize(z_k).
+ * Optional outputs as in orc_encode, with the two margins in place of the two
+ * distances. */
+int orc_encode_polar(const void *W, int w_dtype, int d_out, int d_in, int64_t w_row_stride, int b,
+                     int Ba, int Bp, const float *chan_scale, const int8_t *signs, const float *sigma,
+                     const float *levels, uint8_t *packed, int64_t packed_row_stride, float *row_norm,
+                     float *z_out, int32_t *idx_out, double *margin_a, double *margin_p) {
+    if (d_in % 2 || !is_pow2(b) || b < 2 || d_in % b || Ba < 0 || Bp < 0 || Ba + Bp < 1) return ORC_ERR_ARG;
+    int B = Ba + Bp;
+    int n_pairs = d_in / 2;
+    int64_t row_bytes = orc_packed_row_bytes(d_in, 1 << B);
+    if (packed && packed_row_stride < row_bytes) return ORC_ERR_ARG;
+    size_t esz = w_dtype == 0 ? 4 : 2;
+    int status = ORC_OK;
+#pragma omp parallel
+    {
+        float *y = (float *)malloc(sizeof(float) * (size_t)d_in);
+        int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)n_pairs);
+#pragma omp for schedule(dynamic, 4)
+        for (int i = 0; i < d_out; ++i) {
+            float r;
+            int rc = orc_front_row((const char *)W + (size_t)((int64_t)i * w_row_stride) * esz, w_dtype,
+                                   d_in, b, chan_scale, signs, y, &r);
+            row_norm[i] = r;
+            if (rc != ORC_OK) {
+#pragma omp atomic write
+                status = rc;
+                for (int j = 0; j < d_in; ++j) y[j] = 0.0f;
+            }
+            for (int k = 0; k < n_pairs; ++k) {
+                volatile float q = (float)(1.0 / (double)sigma[k]);
+                volatile float zx = y[2 * k] * q;
+                volatile float zy = y[2 * k + 1] * q;
+                double ma = INFINITY, mp = INFINITY;
+                int a = rc == ORC_OK ? orc_polar_quantize((double)zx, (double)zy, levels, Ba, Bp, &ma, &mp) : 0;
+                idx[k] = a;
+                int64_t o = (int64_t)i * n_pairs + k;
+                if (z_out) {
+                    z_out[2 * o] = zx;
+                    z_out[2 * o + 1] = zy;
+                }
+                if (idx_out) idx_out[o] = a;
+                if (margin_a) margin_a[o] = ma;
+                if (margin_p) margin_p[o] = mp;
+            }
+            if (packed) orc_pack_row(idx, n_pairs, B, packed + (size_t)((int64_t)i * packed_row_stride), row_bytes);
+        }
+        free(y);
+        free(idx);
+    }
+    return status;
+}
