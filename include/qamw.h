@@ -136,6 +136,27 @@ int qamw_status_to_error(int32_t status_word);
 int qamw_codebook_create(const float* codebook_host, int K, int grid, qamw_codebook** out);
 void qamw_codebook_destroy(qamw_codebook* cb);
 
+/* Polar baseline codec (Section 3.5; the corollary on the Rayleigh / uniform-phase source and the
+ * remark on the cut-off R_max = 8).  Amplitude |z_k| / sigma_k goes to the nearest of N_a = 2^Ba
+ * Lloyd-Max levels of the unit Rayleigh density, the phase to one of N_p = 2^Bp uniform bins whose
+ * centres are the odd multiples of pi / N_p; index = (phase << Ba) | amplitude, B = Ba + Bp bits.
+ *
+ * qamw_polar_train: the levels, by Lloyd iterations on the density (centroids from its closed-form
+ * moments on [0, 8]), rounded to f32.  levels_out: host, 2^Ba floats, ascending; c_lm_out (may be
+ * NULL): the normalised distortion C_LM of those f32 levels.  Host only.
+ * qamw_polar_codebook: the 2^(Ba+Bp) reconstruction points level_a (cos phi_p, sin phi_p) as a K x 2
+ * f32 table (host, computed in double, rounded once), i.e. the table that decoding looks up.
+ * qamw_codebook_create_polar: a codebook object for this quantiser on the current device: qamw_decode
+ * uses its K x 2 table like any other codebook; qamw_encode (and qamw_encode_batch) quantise with the
+ * polar rule instead of the nearest-codeword search.  A point on a level threshold takes the lower
+ * level, a point on a bin boundary the bin that starts there, the origin bin 0; results within f32
+ * rounding of a threshold or boundary may fall on either side.  The polar encoder exists only in
+ * the kernels for the common layouts (rows and metadata 32 / 16-byte aligned, d_in a multiple of 16,
+ * 32 <= block <= 512, d_in <= 14336): other shapes get QAMW_ERR_SHAPE. */
+int qamw_polar_train(int Ba, float* levels_out, double* c_lm_out);
+int qamw_polar_codebook(const float* levels, int Ba, int Bp, float* codebook_out);
+int qamw_codebook_create_polar(const float* levels_host, int Ba, int Bp, qamw_codebook** out);
+
 /* Introspection (host values): info_out[0..5] = grid side, total candidate entries, longest
  * candidate list, number of cells with more than four candidates, overflow entries, table bytes. */
 int qamw_codebook_table_info(const qamw_codebook* cb, int32_t* info_out);

@@ -35,6 +35,7 @@ EXPORTED = [
     "qamw_distortion", "qamw_last_cuda_error",
     "qamw_batch_create", "qamw_batch_destroy", "qamw_batch_workspace_bytes", "qamw_calibrate_batch",
     "qamw_encode_batch", "qamw_decode_batch", "qamw_distortion_batch",
+    "qamw_polar_train", "qamw_polar_codebook", "qamw_codebook_create_polar",
 ]
 
 
@@ -93,6 +94,9 @@ def lib() -> C.CDLL:
         L.qamw_decode.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_distortion.argtypes = [vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_last_cuda_error.restype = C.c_char_p
+        L.qamw_polar_train.argtypes = [i32, vp, vp]
+        L.qamw_polar_codebook.argtypes = [vp, i32, i32, vp]
+        L.qamw_codebook_create_polar.argtypes = [vp, i32, i32, C.POINTER(vp)]
         L.qamw_batch_create.argtypes = [C.POINTER(Matrix), i32, vp, C.POINTER(vp)]
         L.qamw_batch_destroy.argtypes = [vp]
         L.qamw_batch_destroy.restype = None
@@ -164,6 +168,21 @@ def status_to_error(status_word: int) -> int:
     return int(lib().qamw_status_to_error(status_word))
 
 
+def polar_train(Ba: int) -> Tuple[np.ndarray, float]:
+    """Lloyd-Max amplitude levels of the polar baseline -> (f32 levels[2^Ba], C_LM)."""
+    lv = np.empty(1 << Ba, np.float32)
+    c = C.c_double()
+    _check("qamw_polar_train", lib().qamw_polar_train(Ba, lv.ctypes.data, C.addressof(c)))
+    return lv, c.value
+
+
+def polar_codebook(levels, Ba: int, Bp: int) -> np.ndarray:
+    lv = _np(levels, np.float32)
+    out = np.empty((1 << (Ba + Bp), 2), np.float32)
+    _check("qamw_polar_codebook", lib().qamw_polar_codebook(lv.ctypes.data, Ba, Bp, out.ctypes.data))
+    return out
+
+
 def search_table_build(codebook, grid: int = 0, budget_bytes: int = 1 << 20):
     """Host-only table construction -> (map f32[4] = zmax, c0, c1, c2; cells u16[grid*grid,4]; overflow u16[];
     info[6])."""
@@ -195,6 +214,18 @@ class Codebook:
         h = C.c_void_p()
         _check("qamw_codebook_create", lib().qamw_codebook_create(cb.ctypes.data, self.K, grid, C.byref(h)))
         self._h = h
+
+    @classmethod
+    def polar(cls, levels, Ba: int, Bp: int) -> "Codebook":
+        """Codebook object of the polar baseline quantiser (qamw_codebook_create_polar)."""
+        lv = _np(levels, np.float32)
+        self = cls.__new__(cls)
+        self.K = 1 << (Ba + Bp)
+        self.host = polar_codebook(lv, Ba, Bp)
+        h = C.c_void_p()
+        _check("qamw_codebook_create_polar", lib().qamw_codebook_create_polar(lv.ctypes.data, Ba, Bp, C.byref(h)))
+        self._h = h
+        return self
 
     @property
     def handle(self):

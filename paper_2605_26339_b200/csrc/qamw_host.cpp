@@ -219,3 +219,76 @@ extern "C" double qamw_bpw(int d_out, int d_in, int K, int has_channel_scales) {
 extern "C" int qamw_status_to_error(int32_t status_word) {
     return (status_word & 1) ? QAMW_ERR_NONFINITE : QAMW_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// polar baseline (Section 3.5): amplitude levels and the table of reconstruction points
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr double kRayleighCutoff = 8.0;  // integration cut-off of the remark after the polar distortion corollary
+
+// Moments int_a^b r^q f(r) dr, q = 0, 1, 2, of the unit Rayleigh density f(r) = r exp(-r^2/2), in
+// closed form (antiderivatives -e, -r e + sqrt(pi/2) erf(r/sqrt 2), -(r^2 + 2) e with e = exp(-r^2/2)).
+void rayleigh_moments(double a, double b, double m[3]) {
+    const double ea = std::exp(-0.5 * a * a), eb = std::exp(-0.5 * b * b);
+    const double root = 1.2533141373155002512078826424055;  // sqrt(pi / 2)
+    m[0] = ea - eb;
+    m[1] = a * ea - b * eb + root * (std::erf(b / 1.4142135623730950488) - std::erf(a / 1.4142135623730950488));
+    m[2] = (a * a + 2.0) * ea - (b * b + 2.0) * eb;
+}
+
+double rayleigh_distortion(const std::vector<double>& l) {
+    const int n = int(l.size());
+    double D = 0.0;
+    for (int j = 0; j < n; ++j) {
+        const double lo = j == 0 ? 0.0 : 0.5 * (l[j - 1] + l[j]);
+        const double hi = j == n - 1 ? kRayleighCutoff : 0.5 * (l[j] + l[j + 1]);
+        double m[3];
+        rayleigh_moments(lo, hi, m);
+        D += m[2] - 2.0 * l[j] * m[1] + l[j] * l[j] * m[0];
+    }
+    return D;
+}
+}  // namespace
+
+extern "C" int qamw_polar_train(int Ba, float* levels_out, double* c_lm_out) {
+    if (!levels_out) return QAMW_ERR_ARG;
+    if (Ba < 0 || Ba > 12) return QAMW_ERR_SHAPE;
+    const int n = 1 << Ba;
+    std::vector<double> l(n), next(n);
+    for (int j = 0; j < n; ++j) l[j] = std::sqrt(-2.0 * std::log(1.0 - (j + 0.5) / n));  // quantiles of the law
+    for (int it = 0; it < 200000; ++it) {
+        double move = 0.0;
+        for (int j = 0; j < n; ++j) {
+            const double lo = j == 0 ? 0.0 : 0.5 * (l[j - 1] + l[j]);
+            const double hi = j == n - 1 ? kRayleighCutoff : 0.5 * (l[j] + l[j + 1]);
+            double m[3];
+            rayleigh_moments(lo, hi, m);
+            next[j] = m[0] > 0.0 ? m[1] / m[0] : l[j];
+            move = std::max(move, std::fabs(next[j] - l[j]));
+        }
+        l.swap(next);
+        if (move < 1e-13) break;
+    }
+    for (int j = 0; j < n; ++j) {
+        levels_out[j] = float(l[j]);
+        l[j] = double(levels_out[j]);
+    }
+    if (c_lm_out) *c_lm_out = rayleigh_distortion(l);
+    return QAMW_OK;
+}
+
+extern "C" int qamw_polar_codebook(const float* levels, int Ba, int Bp, float* codebook_out) {
+    if (!levels || !codebook_out) return QAMW_ERR_ARG;
+    if (Ba < 0 || Bp < 0 || Ba + Bp < 1 || (1 << (Ba + Bp)) > QAMW_MAX_K) return QAMW_ERR_SHAPE;
+    const double pi = 3.14159265358979323846264338327950288;
+    const int Na = 1 << Ba, Np = 1 << Bp;
+    for (int p = 0; p < Np; ++p) {
+        const double phi = (2.0 * p + 1.0) * pi / double(Np);  // bin centres at odd multiples of pi / N_p
+        for (int a = 0; a < Na; ++a) {
+            const int idx = (p << Ba) | a;
+            codebook_out[2 * idx] = float(double(levels[a]) * std::cos(phi));
+            codebook_out[2 * idx + 1] = float(double(levels[a]) * std::sin(phi));
+        }
+    }
+    return QAMW_OK;
+}

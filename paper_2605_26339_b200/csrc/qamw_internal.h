@@ -116,6 +116,10 @@ struct qamw_codebook {
     qamw::CellMap map;
     int n_candidates = 0, max_list = 0, n_overflow_cells = 0;
     std::vector<float> h_codebook;  // host copy (decode only needs the device codebook)
+    // polar baseline: the blob then is [codebook K*2 f32][squared amplitude thresholds 2^Ba f32]
+    // [boundary unit vectors 2^Bp / 2 float2] and off_cells / off_overflow point at the two tables
+    bool polar = false;
+    int polar_ba = 0, polar_bp = 0;
 };
 
 #endif  // QAMW_INTERNAL_H_

@@ -1259,6 +1259,56 @@ extern "C" int qamw_codebook_create(const float* codebook_host, int K, int grid,
     return QAMW_OK;
 }
 
+extern "C" int qamw_codebook_create_polar(const float* levels_host, int Ba, int Bp, qamw_codebook** out) {
+    if (!levels_host || !out) return QAMW_ERR_ARG;
+    *out = nullptr;
+    if (Ba < 0 || Bp < 0 || Ba + Bp < 1 || (1 << (Ba + Bp)) > QAMW_MAX_K) return QAMW_ERR_SHAPE;
+    const int Na = 1 << Ba, Np = 1 << Bp, K = Na * Np;
+    for (int j = 0; j < Na; ++j)
+        if (!(levels_host[j] > 0.f) || (j > 0 && !(levels_host[j] > levels_host[j - 1]))) return QAMW_ERR_ARG;
+    qamw_codebook* cb = new (std::nothrow) qamw_codebook();
+    if (!cb) return QAMW_ERR_NOMEM;
+    cb->K = K;
+    cb->polar = true;
+    cb->polar_ba = Ba;
+    cb->polar_bp = Bp;
+    cb->h_codebook.resize(size_t(2) * K);
+    qamw_polar_codebook(levels_host, Ba, Bp, cb->h_codebook.data());
+    // squared thresholds between adjacent levels (the last entry is never read), then the unit vectors
+    // of the bin boundaries 2 pi k / N_p of the upper half plane
+    const int n_bnd = std::max(1, Np / 2);
+    const int n_thr = std::max(2, Na);  // an even count keeps the 8-byte vectors behind it aligned
+    std::vector<float> tables(size_t(n_thr) + 2 * size_t(n_bnd), 0.f);
+    for (int j = 0; j + 1 < Na; ++j) {
+        const double t = 0.5 * (double(levels_host[j]) + double(levels_host[j + 1]));
+        tables[j] = float(t * t);
+    }
+    tables[Na - 1] = INFINITY;
+    const double pi = 3.14159265358979323846264338327950288;
+    for (int k2 = 0; k2 < n_bnd; ++k2) {
+        const double beta = 2.0 * pi * k2 / double(Np);
+        tables[n_thr + 2 * k2] = float(std::cos(beta));
+        tables[n_thr + 2 * k2 + 1] = float(std::sin(beta));
+    }
+    cb->off_cells = size_t(K) * 8;
+    cb->off_overflow = cb->off_cells + size_t(n_thr) * 4;
+    cb->blob_bytes = (cb->off_cells + tables.size() * 4 + 15) & ~size_t(15);
+    std::vector<unsigned char> blob(cb->blob_bytes, 0);
+    std::memcpy(blob.data(), cb->h_codebook.data(), size_t(K) * 8);
+    std::memcpy(blob.data() + cb->off_cells, tables.data(), tables.size() * 4);
+    cudaError_t e = cudaGetDevice(&cb->device);
+    if (e == cudaSuccess) e = cudaMalloc(&cb->d_blob, cb->blob_bytes);
+    if (e == cudaSuccess) e = cudaMemcpy(cb->d_blob, blob.data(), cb->blob_bytes, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        set_cuda_error("qamw_codebook_create_polar", int(e));
+        if (cb->d_blob) cudaFree(cb->d_blob);
+        delete cb;
+        return QAMW_ERR_CUDA;
+    }
+    *out = cb;
+    return QAMW_OK;
+}
+
 extern "C" void qamw_codebook_destroy(qamw_codebook* cb) {
     if (!cb) return;
     if (cb->d_blob) cudaFree(cb->d_blob);
@@ -1303,6 +1353,7 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
                          status_out, stream);
         if (rc != QAMW_ERR_SHAPE) return rc;
     }
+    if (cb->polar) return QAMW_ERR_SHAPE;  // the polar quantiser exists in the kernels for the common layouts only
     EncodeArgs a;
     a.g = make_geom(p, W);
     a.g.cvec = const_vec_ok(p, chan_scale, signs, sigma);

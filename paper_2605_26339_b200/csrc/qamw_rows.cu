@@ -394,7 +394,44 @@ struct Encode2Args {
     int brute;
     float inv_sqrt_b;        // c_b = f32(1 / sqrt(b))
     int32_t* status;         // out (optional): bit 0 set when a row norm is not finite
+    int polar_ba, polar_bp;  // polar quantiser: amplitude and phase bits; `table` then holds the squared
+                             // amplitude thresholds (2^Ba floats) and, from off_overflow on, the unit vectors
+                             // of the phase bin boundaries of the upper half plane (2^Bp / 2 float2)
 };
+
+// Polar quantiser (Section 3.5): amplitude |z| to the nearest of 2^Ba levels, phase to one of 2^Bp
+// uniform bins, index = (phase << Ba) | amplitude.  Both are binary searches over small tables in
+// shared memory: squared thresholds (midpoints of adjacent levels) for the amplitude, and for the
+// phase the sign of the cross product with the boundary directions after folding the lower half plane
+// onto the upper one.  A point on a threshold takes the lower level, a point on a boundary the bin
+// that starts there, the origin bin 0 -- the oracle's rules; within f32 rounding of a threshold or a
+// boundary either neighbour may come out.
+struct PolarSmem {
+    uint32_t thr2;  // shared-memory address of the squared thresholds
+    uint32_t bnd;   // ... of the boundary unit vectors
+    int Ba, Bp;
+};
+__device__ __forceinline__ int search_polar(const PolarSmem& s, float zx, float zy) {
+    const float r2 = __fmaf_rn(zy, zy, __fmul_rn(zx, zx));
+    int a = 0;
+    for (int step = (1 << s.Ba) >> 1; step > 0; step >>= 1) {
+        float t;
+        asm("ld.shared.f32 %0, [%1];" : "=f"(t) : "r"(s.thr2 + 4u * uint32_t(a + step - 1)));
+        if (r2 > t) a += step;
+    }
+    int p = 0;
+    if (s.Bp > 0) {
+        const bool lower = zy < 0.f || (zy == 0.f && zx < 0.f);
+        const float x = lower ? -zx : zx, y = lower ? -zy : zy;
+        for (int step = (1 << s.Bp) >> 2; step > 0; step >>= 1) {
+            const float2 b = lds_f32x2(s.bnd + 8u * uint32_t(p + step));
+            if (__fmaf_rn(b.x, y, -__fmul_rn(b.y, x)) >= 0.f) p += step;
+        }
+        if (lower) p += (1 << s.Bp) >> 1;
+        if (r2 == 0.f) p = 0;
+    }
+    return (p << s.Ba) | a;
+}
 
 // Index staging of a warp: its 64 octets as one 64-bit value each (index p of the octet at bits
 // [p B, (p+1) B)); 8 slots of padding after every 16 keep the two stores of a warp on distinct banks
@@ -409,7 +446,7 @@ struct Stage2 {
 // adds up its part of the row norm, rotates (shuffles only), and after the one meeting point of the
 // row's warps -- a named barrier for the norm -- searches its 256 pairs, stages the indices and
 // writes its 32 B bytes of the packed row.  W is read once.
-template <bool BF16, int LOG2B, int NS, int MAXT>
+template <bool BF16, int LOG2B, int NS, int MAXT, bool POLAR>
 __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
     constexpr int WE = 256 * NS;
     typedef Lay2<NS, LOG2B> Lay;
@@ -418,8 +455,8 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
     __shared__ MatDesc cur;            // the matrix the block is working on (re-read per row: saves registers)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
 
-    const int cb_bytes = (a.K * 8) << a.log2c;
-    fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
+    const int cb_bytes = POLAR ? 0 : (a.K * 8) << a.log2c;  // the polar quantiser never reads codewords
+    if (!POLAR) fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
     unsigned char* table = smem + cb_bytes;
     {
         uint4* dst = reinterpret_cast<uint4*>(table);
@@ -453,6 +490,11 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
     s.c1 = pack2(a.map_c1, a.map_c1);
     s.c2 = pack2(a.map_c2, a.map_c2);
     s.bias = pack2(a.map_bias, a.map_bias);
+    PolarSmem ps;
+    ps.thr2 = smem_addr(table);
+    ps.bnd = smem_addr(table + a.off_overflow);
+    ps.Ba = a.polar_ba;
+    ps.Bp = a.polar_bp;
 
     const int B = a.log2K, B4 = 4 * a.log2K;
     const unsigned div_magic = 0xffffffffu / unsigned(B4) + 1u;  // ceil(2^32 / (4B))
@@ -521,7 +563,7 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
         double* part_base = &ss_part[0][group * n_seg];
 
         auto rows = [&](auto mode_tag) {
-            constexpr int MODE = decltype(mode_tag)::value;  // 0 = table, 1 = table with reach check, 2 = exhaustive
+            constexpr int MODE = decltype(mode_tag)::value;  // 0 = table, 1 = table with reach check, 2 = exhaustive, 3 = polar
             int parity = 0;
             // raw bits of the thread's elements of one row; the next row is fetched as soon as this one
             // has been converted, so its latency hides behind the rotation and the search
@@ -599,7 +641,10 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
                         unpack2(mul2(P[p][i], gn2), yx, yy);
                         z[i] = make_float2(__fmul_rn(yx, q[p][i]), __fmul_rn(yy, q[p][i]));
                     }
-                    if (MODE == 0) {
+                    if (MODE == 3) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) v[i] = uint32_t(search_polar(ps, z[i].x, z[i].y));
+                    } else if (MODE == 0) {
                         uint2 rec[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) v[i] = uint32_t(search_cell(s, z[i].x, z[i].y, rec[i]));
@@ -654,9 +699,13 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
                 __syncwarp();  // the staging piece is free again
             }
         };
-        if (a.brute) rows(std::integral_constant<int, 2>{});
-        else if (any_risky) rows(std::integral_constant<int, 1>{});
-        else rows(std::integral_constant<int, 0>{});
+        if constexpr (POLAR) {
+            rows(std::integral_constant<int, 3>{});
+        } else {
+            if (a.brute) rows(std::integral_constant<int, 2>{});
+            else if (any_risky) rows(std::integral_constant<int, 1>{});
+            else rows(std::integral_constant<int, 0>{});
+        }
     }
 }
 
@@ -712,13 +761,19 @@ int launch_decode2(const Decode2Args& a, int blocks, int threads, size_t smem, c
 
 template <bool BF16, int LOG2B, int NS, int MAXT>
 int launch_encode2(const Encode2Args& a, int blocks, int threads, size_t smem, cudaStream_t st) {
-    int rc = raise_smem_limit(reinterpret_cast<const void*>(&encode2_kernel<BF16, LOG2B, NS, MAXT>));
+    if (a.polar_ba >= 0) {
+        int rc = raise_smem_limit(reinterpret_cast<const void*>(&encode2_kernel<BF16, LOG2B, NS, MAXT, true>));
+        if (rc) return rc;
+        encode2_kernel<BF16, LOG2B, NS, MAXT, true><<<blocks, threads, smem, st>>>(a);
+        return launch_check("encode2_kernel (polar)");
+    }
+    int rc = raise_smem_limit(reinterpret_cast<const void*>(&encode2_kernel<BF16, LOG2B, NS, MAXT, false>));
     if (rc) return rc;
-    encode2_kernel<BF16, LOG2B, NS, MAXT><<<blocks, threads, smem, st>>>(a);
+    encode2_kernel<BF16, LOG2B, NS, MAXT, false><<<blocks, threads, smem, st>>>(a);
     return launch_check("encode2_kernel");
 }
 
-constexpr size_t kEncode2StaticSmem = 512;  // ss_part
+constexpr size_t kEncode2StaticSmem = 1024;  // ss_part and the current matrix descriptor, rounded up
 
 }  // namespace
 
@@ -857,10 +912,12 @@ int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, cons
     a.brute = (flags & QAMW_FLAG_BRUTE_FORCE) ? 1 : 0;
     a.inv_sqrt_b = float(1.0 / std::sqrt(double(block)));
     a.status = status;
+    a.polar_ba = cb->polar ? cb->polar_ba : -1;
+    a.polar_bp = cb->polar ? cb->polar_bp : -1;
     const size_t fixed = ((size_t(a.table_bytes) + 15) & ~size_t(15)) + size_t(warps) * Stage2<NS>::kSlots * 8;
     if (fixed + size_t(K) * 8 > kSmemLimit - kEncode2StaticSmem) return QAMW_ERR_SHAPE;
-    a.log2c = pick_copies(K, kSmemLimit - kEncode2StaticSmem - fixed);
-    const size_t smem = fixed + (size_t(K) * 8 << a.log2c);
+    a.log2c = cb->polar ? 0 : pick_copies(K, kSmemLimit - kEncode2StaticSmem - fixed);
+    const size_t smem = fixed + (cb->polar ? 0 : (size_t(K) * 8 << a.log2c));
     int grid = sm_count();
     if (flags & QAMW_FLAG_HALF_DEVICE) grid = std::max(1, grid / 2);
     const int blocks = spans_dev ? span_blocks : int(std::max<long long>(1, std::min<long long>(grid, rows)));

@@ -482,3 +482,69 @@ def test_batch_equals_single_matrix_calls(orc, shapes, block):
     exempt = (enc["d2_second"] - enc["d2_best"]) < 1e-6 * enc["d2_second"]
     assert not np.any((idx != enc["idx"]) & ~exempt)
     assert np.array_equal(s0["norm"].cpu().numpy(), enc["row_norm"])
+
+
+@pytest.mark.parametrize("Ba,Bp,d_out,d_in,block,dtype", [
+    (5, 6, 48, 2048, 128, torch.bfloat16),   # the paper's 11-bit split
+    (3, 4, 33, 1024, 64, torch.float32),
+    (0, 3, 9, 512, 32, torch.bfloat16),      # phase only
+    (4, 0, 9, 512, 256, torch.bfloat16),     # amplitude only
+    (5, 6, 20, 13824, 128, torch.bfloat16),  # the longest rows of configuration 3
+])
+def test_polar_baseline_codec(orc, Ba, Bp, d_out, d_in, block, dtype):
+    """Polar baseline (Section 3.5) on the GPU against the oracle: indices equal except where the
+    oracle's margins say that f32 cannot tell (amplitude within 1e-6 relative of a level threshold,
+    phase within 1e-6 rad of a bin boundary) -- there the GPU's index must be the neighbouring level
+    or bin; decode of the oracle's stream through the reconstruction table as for the 2-D codec."""
+    W, act = _make(d_out, d_in, dtype, 700 + Ba * 16 + Bp)
+    W[1] = 0  # a zero row: every pair is the origin (phase bin 0, lowest level)
+    lv, _ = q.polar_train(Ba)
+    cb = q.Codebook.polar(lv, Ba, Bp)
+    K, B = 1 << (Ba + Bp), Ba + Bp
+    s = q.channel_scales(act, 0.3)
+    signs = q.make_signs(q.DEFAULT_SIGN_SEED, d_in)
+    Wd, s_d, signs_d = W.to(DEV), torch.from_numpy(s).to(DEV), torch.from_numpy(signs).to(DEV)
+    sigma, _ = orc.calibrate(_to_bits(Wd), block, s, signs)
+    sigma_d = torch.from_numpy(sigma).to(DEV)
+    p = q.make_params(Wd, d_out, d_in, block, K, 0, (q.packed_row_bytes(d_in, K) + 15) // 16 * 16)
+    packed = torch.full((d_out, p.packed_row_stride), 0xEE, dtype=torch.uint8, device=DEV)
+    norm = torch.empty(d_out, dtype=torch.float32, device=DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    q.encode(Wd, p, s_d, signs_d, sigma_d, cb, packed, norm, st)
+    enc = orc.encode_polar(_to_bits(Wd), block, lv, Ba, Bp, s, signs, sigma, packed_row_stride=p.packed_row_stride,
+                           diagnostics=True)
+    torch.cuda.synchronize()
+    assert int(st.cpu()[0]) == 0 and np.array_equal(norm.cpu().numpy(), enc["row_norm"])
+    pk = packed.cpu().numpy()
+    idx = np.stack([orc.unpack_row(r, d_in // 2, B) for r in pk])
+    diff = idx != enc["idx"]
+    exempt = (enc["margin_a"] < 1e-6) | (enc["margin_p"] < 1e-6)
+    assert not np.any(diff & ~exempt), f"{int((diff & ~exempt).sum())} non-exempt index mismatches"
+    if diff.any():  # one step in the ambiguous component only
+        ga, gp = idx[diff] & ((1 << Ba) - 1), idx[diff] >> Ba
+        oa, op = enc["idx"][diff] & ((1 << Ba) - 1), enc["idx"][diff] >> Ba
+        dp = np.abs(gp - op)
+        assert np.all(np.abs(ga - oa) <= 1) and np.all((dp <= 1) | (dp == (1 << Bp) - 1))
+    assert not idx[1].any()
+    rb = q.packed_row_bytes(d_in, K)
+    assert not pk[:, rb:].any()
+    # decode the oracle's stream
+    what = torch.empty((d_out, d_in), dtype=torch.bfloat16, device=DEV)
+    q.decode(torch.from_numpy(enc["packed"]).to(DEV), torch.from_numpy(enc["row_norm"]).to(DEV), s_d, signs_d, sigma_d, cb, p, what)
+    ref = orc.decode(enc["packed"], enc["row_norm"], block, cb.host, s, signs, sigma, d_in)
+    ulps = np.abs(_bf16_ordered(_to_bits(what)) - _bf16_ordered(ref))
+    assert (ulps <= 1).mean() > 1 - kFarFraction - 2.0 / ulps.size and (ulps == 0).mean() > 0.98
+    print("PARITY polar", dict(Ba=Ba, Bp=Bp, pairs=int(idx.size), mismatches=int(diff.sum()), exempt=int(exempt.sum())))
+
+
+def test_polar_encoder_refuses_layouts_outside_its_kernels(orc):
+    lv, _ = q.polar_train(2)
+    cb = q.Codebook.polar(lv, 2, 2)
+    W = torch.zeros((4, 64), dtype=torch.float32, device=DEV)
+    p = q.make_params(W, 4, 64, 16, 16)  # block 16: only the general kernels take it
+    dummy = torch.zeros(64, dtype=torch.uint8, device=DEV)
+    signs = torch.ones(64, dtype=torch.int8, device=DEV)
+    sigma = torch.ones(32, dtype=torch.float32, device=DEV)
+    with pytest.raises(q.QamwError) as e:
+        q.encode(W, p, None, signs, sigma, cb, dummy, sigma)
+    assert e.value.code == q.ERR_SHAPE

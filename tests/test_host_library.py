@@ -199,3 +199,23 @@ def test_argument_errors_are_reported_before_any_launch():
     assert q.packed_row_bytes(255, 256) == 0 and q.block_size_rule(0) == 0
     with pytest.raises(q.QamwError):
         q.make_signs(1, 0)
+
+
+@pytest.mark.parametrize("Ba", [0, 1, 3, 5])
+def test_polar_levels_and_table_agree_with_oracle(orc, Ba):
+    """The library's Rayleigh Lloyd-Max levels (closed-form moments) against the oracle's (Simpson
+    quadrature): two implementations of Section 3.5's amplitude quantiser.  Lloyd's iteration creeps
+    towards its fixed point, so the levels agree to the stopping tolerances and the distortion, which
+    is flat there, far more closely.  Given the same levels the reconstruction tables are identical."""
+    lv, c = q.polar_train(Ba)
+    lo, co = orc.rayleigh_lloyd_max(1 << Ba)
+    assert np.allclose(lv, lo, atol=1e-5) and abs(c - co) < 1e-9
+    assert np.array_equal(q.polar_codebook(lv, Ba, 4), orc.polar_codebook(lv, Ba, 4))
+    lib = q.lib()
+    h = C.c_void_p()
+    assert lib.qamw_polar_train(13, lv.ctypes.data, None) == q.ERR_SHAPE
+    assert lib.qamw_polar_train(2, None, None) == q.ERR_ARG
+    assert lib.qamw_polar_codebook(lv.ctypes.data, 7, 6, lv.ctypes.data) == q.ERR_SHAPE  # more than 4096 points
+    assert lib.qamw_codebook_create_polar(None, 2, 2, C.byref(h)) == q.ERR_ARG
+    bad = np.array([1.0, 0.5], np.float32)  # not ascending
+    assert lib.qamw_codebook_create_polar(bad.ctypes.data, 1, 2, C.byref(h)) == q.ERR_ARG
