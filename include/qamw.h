@@ -97,6 +97,24 @@ typedef struct qamw_codebook qamw_codebook; /* opaque: device copy of C plus its
 int qamw_train_codebook(int K, uint64_t n_samples, uint64_t seed, int max_iters, double rel_tol,
                         float* codebook_out, double* train_mse_out);
 
+/* The same training on the current CUDA device (Section 3.6; the paper's Limitations section puts
+ * its own trainer at about 5 s per bitrate level and names per-checkpoint codebooks as follow-up).
+ * Same rules as qamw_train_codebook: same initial codewords, exact assignment in double (every
+ * sample against every codeword, d = dx*dx + dy*dy with one rounding per operation, lowest index on
+ * ties), every cell's samples added in sample order, same stopping rule, same final order and f32
+ * rounding; the result does not vary from run to run.
+ * samples_dev: device, n_samples (x, y) pairs of doubles to train on -- e.g. normalised pairs of a
+ * checkpoint -- or NULL: the unit circular Gaussian samples of counter stream `seed` are generated on
+ * the device (the device's log / sin / cos may differ from the host's in the last bit).
+ * codebook_out: host, K*2 floats.  Optional host outputs (NULL to skip): train_mse_out as in
+ * qamw_train_codebook; iters_out: centroid updates done; mse_trace_out: max_iters + 1 doubles, the
+ * mean squared distance before every update; seconds_out: wall time of the call.
+ * Synchronous; allocates and frees its device scratch (about 32 bytes per sample) itself.
+ * n_samples < 2^31. */
+int qamw_train_codebook_gpu(int K, uint64_t n_samples, uint64_t seed, const double* samples_dev, int max_iters,
+                            double rel_tol, float* codebook_out, double* train_mse_out, int* iters_out,
+                            double* mse_trace_out, double* seconds_out);
+
 /* Section B.2: s_j = clamp(r_j^alpha / geomean(r^alpha), 1/16, 16); r_j floored at FLT_MIN;
  * alpha == 0 gives all ones.  act_rms, s_out: host, d_in floats. */
 int qamw_channel_scales(const float* act_rms, int d_in, float alpha, float* s_out);

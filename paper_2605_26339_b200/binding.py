@@ -35,7 +35,7 @@ EXPORTED = [
     "qamw_distortion", "qamw_last_cuda_error",
     "qamw_batch_create", "qamw_batch_destroy", "qamw_batch_workspace_bytes", "qamw_calibrate_batch",
     "qamw_encode_batch", "qamw_decode_batch", "qamw_distortion_batch",
-    "qamw_polar_train", "qamw_polar_codebook", "qamw_codebook_create_polar",
+    "qamw_train_codebook_gpu", "qamw_polar_train", "qamw_polar_codebook", "qamw_codebook_create_polar",
 ]
 
 
@@ -94,6 +94,7 @@ def lib() -> C.CDLL:
         L.qamw_decode.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_distortion.argtypes = [vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_last_cuda_error.restype = C.c_char_p
+        L.qamw_train_codebook_gpu.argtypes = [i32, u64, u64, vp, i32, C.c_double, vp, vp, vp, vp, vp]
         L.qamw_polar_train.argtypes = [i32, vp, vp]
         L.qamw_polar_codebook.argtypes = [vp, i32, i32, vp]
         L.qamw_codebook_create_polar.argtypes = [vp, i32, i32, C.POINTER(vp)]
@@ -137,6 +138,23 @@ def train_codebook(K: int, n_samples: int = 1 << 20, seed: int = 0, max_iters: i
     _check("qamw_train_codebook", lib().qamw_train_codebook(K, n_samples, seed, max_iters, rel_tol,
                                                            cb.ctypes.data, C.addressof(mse)))
     return cb, mse.value
+
+
+def train_codebook_gpu(K: int, n_samples: int = 1 << 20, seed: int = 0, max_iters: int = 100, rel_tol: float = 1e-6,
+                       samples: Optional[torch.Tensor] = None):
+    """Lloyd training on the current CUDA device -> dict(codebook, mse, iters, trace, seconds).
+    samples: optional float64 device tensor [n, 2] to train on instead of the generated Gaussian."""
+    cb = np.empty((K, 2), np.float32)
+    mse, secs, iters = C.c_double(), C.c_double(), C.c_int()
+    trace = np.full(max_iters + 2, np.nan, np.float64)
+    if samples is not None:
+        if samples.dtype != torch.float64 or samples.dim() != 2 or samples.shape[1] != 2 or not samples.is_contiguous():
+            raise TypeError("samples must be a contiguous float64 [n, 2] device tensor")
+        n_samples = samples.shape[0]
+    _check("qamw_train_codebook_gpu", lib().qamw_train_codebook_gpu(
+        K, n_samples, seed, _dp(samples), max_iters, rel_tol, cb.ctypes.data, C.addressof(mse), C.addressof(iters),
+        trace.ctypes.data, C.addressof(secs)))
+    return dict(codebook=cb, mse=mse.value, iters=iters.value, trace=trace[~np.isnan(trace)], seconds=secs.value)
 
 
 def channel_scales(act_rms, alpha: float) -> np.ndarray:
