@@ -369,3 +369,23 @@ def encode_polar(W, b, levels, Ba, Bp, chan_scale, signs, sigma, packed_row_stri
                                 _p(_c(signs, np.int8)), _p(_c(sigma, np.float32)), _p(lv), _p(packed), C.c_int64(stride),
                                 _p(norms), _p(z), _p(idx), _p(ma), _p(mp))
     return dict(status=int(rc), packed=packed, row_norm=norms, z=z, idx=idx, margin_a=ma, margin_p=mp)
+
+
+# ------------------------------------------------------------------------------- variants
+def round_f16(values) -> np.ndarray:
+    v = np.array(values, np.float32, copy=True).ravel()
+    lib().orc_round_f16(_p(v), C.c_int64(v.shape[0]))
+    return v.reshape(np.shape(values))
+
+
+def renorm_row_norms(packed, row_norm, sigma, codebook, d_in) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, np.uint8)
+    d_out, stride = packed.shape
+    cb = _c(codebook, np.float32)
+    out = np.empty(d_out, np.float32)
+    rc = lib().orc_renorm_row_norms(_p(packed), C.c_int64(stride), _p(_c(row_norm, np.float32)),
+                                    _p(_c(sigma, np.float32)), _p(cb), C.c_int(cb.shape[0]), C.c_int(d_out),
+                                    C.c_int(d_in), _p(out))
+    if rc != ORC_OK:
+        raise ValueError(f"orc_renorm_row_norms failed: {rc}")
+    return out

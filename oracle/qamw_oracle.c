@@ -848,3 +848,50 @@ int orc_encode_polar(const void *W, int w_dtype, int d_out, int d_in, int64_t w_
     }
     return status;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Variants around the path.                                                   */
+/* ------------------------------------------------------------------------- */
+
+/* Section 3.2: "a fully serialized f16 row norm" -- metadata rounded to IEEE
+ * binary16 (nearest even; overflow to infinity, gradual underflow) and widened
+ * back to f32, in place. */
+void orc_round_f16(float *v, int64_t n) {
+    for (int64_t i = 0; i < n; ++i) {
+        double x = (double)v[i];
+        if (x != x || x == INFINITY || x == -INFINITY || x == 0.0) continue;
+        double a = fabs(x);
+        int e;
+        frexp(a, &e); /* a = m 2^e, m in [0.5, 1) */
+        int q = e - 11; /* spacing 2^q: 11 significant bits */
+        if (q < -24) q = -24; /* subnormal spacing 2^-24 */
+        double r = nearbyint(ldexp(a, -q)); /* ties to even in the default rounding mode */
+        double y = ldexp(r, q);
+        if (y >= 65520.0) y = INFINITY; /* beyond the largest finite half (65504) after rounding */
+        v[i] = (float)(x < 0 ? -y : y);
+    }
+}
+
+/* Section A.3, optional final direction renormalisation: the decoder divides the
+ * reconstructed direction by its own length before multiplying by the stored row
+ * norm.  The rotation preserves lengths (Lemma 1), so that length is
+ * |yhat| = sqrt(sum_k sigma_k^2 |c_idx_k|^2); out[i] = f32(r_i / |yhat_i|) is the
+ * factor to hand to the decoder in place of r_i (0 for an all-zero yhat). */
+int orc_renorm_row_norms(const uint8_t *packed, int64_t packed_row_stride, const float *row_norm,
+                         const float *sigma, const float *codebook, int K, int d_out, int d_in, float *out) {
+    if (d_in % 2 || !is_pow2(K)) return ORC_ERR_ARG;
+    int B = ilog2(K), n_pairs = d_in / 2;
+    int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)n_pairs);
+    for (int i = 0; i < d_out; ++i) {
+        orc_unpack_row(packed + (size_t)((int64_t)i * packed_row_stride), n_pairs, B, idx);
+        double ss = 0.0;
+        for (int k = 0; k < n_pairs; ++k) {
+            double cx = (double)codebook[2 * idx[k]] * (double)sigma[k];
+            double cy = (double)codebook[2 * idx[k] + 1] * (double)sigma[k];
+            ss += cx * cx + cy * cy;
+        }
+        out[i] = ss > 0.0 ? (float)((double)row_norm[i] / sqrt(ss)) : 0.0f;
+    }
+    free(idx);
+    return ORC_OK;
+}
