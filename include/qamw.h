@@ -251,6 +251,19 @@ int qamw_decode(const uint8_t* packed, const float* row_norm, const float* chan_
                 const int8_t* signs, const float* sigma, const qamw_codebook* cb, const qamw_params* p,
                 void* w_hat_bf16_out, void* stream);
 
+/* Variants around the path.
+ * qamw_round_f16 (Section 3.2: the bitrate charges 16 bits per row norm and per channel scale; "a
+ * fully serialized f16 row norm" adds a radial quantisation term): rounds n f32 values on the device,
+ * in place, to IEEE binary16 (nearest even) and back.  Round channel scales and sigma before
+ * qamw_encode, row norms after it, and decode sees exactly what a 16-bit serialisation would hold.
+ * qamw_renorm_row_norms (Section A.3, the optional final direction renormalisation): writes
+ * row_norm_out[i] = r_i / |yhat_i|, |yhat_i|^2 = sum_k sigma_k^2 |c_idx_k|^2 (the rotation preserves
+ * lengths, Lemma 1); decoding with these factors in place of the row norms gives rows whose scaled
+ * length is r_i again.  row_norm_out may alias row_norm.  Both asynchronous on `stream`. */
+int qamw_round_f16(float* values, size_t n, void* stream);
+int qamw_renorm_row_norms(const uint8_t* packed, const float* row_norm, const float* sigma, const qamw_codebook* cb,
+                          const qamw_params* p, float* row_norm_out, void* stream);
+
 /* Corollary 3 / Corollary 4 sums in double:
  *   out4[0] = sum (W - W_hat)^2        out4[1] = sum W^2
  *   out4[2] = sum r_j^2 (W - W_hat)^2  out4[3] = sum r_j^2 W^2     (r_j = act_rms, 1 if NULL)

@@ -35,7 +35,7 @@ EXPORTED = [
     "qamw_distortion", "qamw_last_cuda_error",
     "qamw_batch_create", "qamw_batch_destroy", "qamw_batch_workspace_bytes", "qamw_calibrate_batch",
     "qamw_encode_batch", "qamw_decode_batch", "qamw_distortion_batch",
-    "qamw_train_codebook_gpu", "qamw_polar_train", "qamw_polar_codebook", "qamw_codebook_create_polar",
+    "qamw_train_codebook_gpu", "qamw_round_f16", "qamw_renorm_row_norms", "qamw_polar_train", "qamw_polar_codebook", "qamw_codebook_create_polar",
 ]
 
 
@@ -95,6 +95,8 @@ def lib() -> C.CDLL:
         L.qamw_distortion.argtypes = [vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_last_cuda_error.restype = C.c_char_p
         L.qamw_train_codebook_gpu.argtypes = [i32, u64, u64, vp, i32, C.c_double, vp, vp, vp, vp, vp]
+        L.qamw_round_f16.argtypes = [vp, sz, vp]
+        L.qamw_renorm_row_norms.argtypes = [vp, vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_polar_train.argtypes = [i32, vp, vp]
         L.qamw_polar_codebook.argtypes = [vp, i32, i32, vp]
         L.qamw_codebook_create_polar.argtypes = [vp, i32, i32, C.POINTER(vp)]
@@ -343,6 +345,19 @@ def decode(packed: torch.Tensor, row_norm: torch.Tensor, chan_scale, signs, sigm
            w_hat_out: torch.Tensor, stream=None):
     _check("qamw_decode", lib().qamw_decode(_dp(packed), _dp(row_norm), _dp(chan_scale), _dp(signs), _dp(sigma),
                                            cb.handle, C.byref(p), _dp(w_hat_out), _stream(stream)))
+
+
+def round_f16(values: torch.Tensor, stream=None):
+    """Rounds a float32 device tensor in place to what a 16-bit (f16) serialisation would hold."""
+    if values.dtype != torch.float32 or not values.is_contiguous():
+        raise TypeError("values must be a contiguous float32 tensor")
+    _check("qamw_round_f16", lib().qamw_round_f16(_dp(values), values.numel(), _stream(stream)))
+
+
+def renorm_row_norms(packed: torch.Tensor, row_norm: torch.Tensor, sigma, cb: Codebook, p: Params,
+                     row_norm_out: torch.Tensor, stream=None):
+    _check("qamw_renorm_row_norms", lib().qamw_renorm_row_norms(_dp(packed), _dp(row_norm), _dp(sigma), cb.handle,
+                                                               C.byref(p), _dp(row_norm_out), _stream(stream)))
 
 
 def distortion(W: torch.Tensor, w_hat: torch.Tensor, act_rms, p: Params, out4: torch.Tensor, stream=None):

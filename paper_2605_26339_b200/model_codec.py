@@ -39,6 +39,37 @@ def combine_distortion(sums4: torch.Tensor, n_weights: int, group=None) -> Dict[
             "mse": float(d[0] / d[4]), "n_weights": int(d[4])}
 
 
+def choose_alpha(W: torch.Tensor, act_rms: torch.Tensor, codebook: q.Codebook, block: int,
+                 grid=(0.0, 0.3, 0.5, 0.8), sign_seed: int = q.DEFAULT_SIGN_SEED):
+    """Scaling exponent for one matrix from the paper's grid {0, 0.3, 0.5, 0.8} (Section B.2 and the
+    hyper-parameter table): every candidate goes through channel scales -> calibrate -> encode ->
+    decode, and the one with the smallest diagonal-M_x relative output error rho_o (Corollary 4) wins.
+    Returns (best alpha, {alpha: (rho_w, rho_o)})."""
+    dev = W.device
+    d_out, d_in = W.shape
+    K = codebook.K
+    p = q.make_params(W, d_out, d_in, block, K)
+    signs = torch.from_numpy(q.make_signs(sign_seed, d_in)).to(dev)
+    sigma = torch.empty(d_in // 2, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(8, q.calibrate_workspace_bytes(p)), dtype=torch.uint8, device=dev)
+    packed = torch.empty((d_out, p.packed_row_stride), dtype=torch.uint8, device=dev)
+    norm = torch.empty(d_out, dtype=torch.float32, device=dev)
+    w_hat = torch.empty((d_out, d_in), dtype=torch.bfloat16, device=dev)
+    out4 = torch.empty(4, dtype=torch.float64, device=dev)
+    act_host = act_rms.detach().cpu().numpy()
+    scores = {}
+    for alpha in grid:
+        s = torch.from_numpy(q.channel_scales(act_host, alpha)).to(dev) if alpha else None
+        q.calibrate(W, p, s, signs, sigma, ws)
+        q.encode(W, p, s, signs, sigma, codebook, packed, norm)
+        q.decode(packed, norm, s, signs, sigma, codebook, p, w_hat)
+        q.distortion(W, w_hat, act_rms, p, out4)
+        d = out4.cpu().numpy()
+        scores[float(alpha)] = (float(np.sqrt(d[0] / d[1])), float(np.sqrt(d[2] / d[3])))
+    best = min(scores, key=lambda a: scores[a][1])
+    return best, scores
+
+
 @dataclass
 class MatrixSlot:
     """Device-resident state of one weight matrix."""
