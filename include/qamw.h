@@ -45,7 +45,7 @@ extern "C" {
 
 #define QAMW_OK 0
 #define QAMW_ERR_ARG (-1)       /* NULL pointer, value out of range */
-#define QAMW_ERR_SHAPE (-2)     /* d_in odd, block does not divide d_in, K / block not a power of two */
+#define QAMW_ERR_SHAPE (-2)     /* d_in odd or above 16384, block does not divide d_in, K / block not a power of two */
 #define QAMW_ERR_ALIGN (-3)     /* pointer or stride alignment */
 #define QAMW_ERR_CUDA (-4)      /* a CUDA runtime call failed */
 #define QAMW_ERR_NONFINITE (-5) /* reported by qamw_status_to_error for a non-finite row norm */
@@ -70,7 +70,7 @@ extern "C" {
 #define QAMW_STATIC_SCRATCH_BYTES (16u << 20) /* built-in scratch of qamw_calibrate_static */
 
 typedef struct {
-    int32_t d_out, d_in;       /* d_in even, block | d_in */
+    int32_t d_out, d_in;       /* d_in even, block | d_in, d_in <= 16384 (a row is held by one thread block) */
     int32_t block;             /* b = 2^q, 2 <= b <= 1024 */
     int32_t K;                 /* codebook size, power of two, 2 <= K <= 4096 */
     int32_t w_dtype;           /* QAMW_DTYPE_* of W */
@@ -234,12 +234,27 @@ int qamw_calibrate(const void* W, const qamw_params* p, const float* chan_scale,
 int qamw_calibrate_static(const void* W, const qamw_params* p, const float* chan_scale, const int8_t* signs,
                           float* sigma_out, int32_t* status_out, void* stream);
 
-/* Section 3.1 steps 1-6 (after Section B.2 scaling) for all rows.  Writes packed_out
+/* Section 3.1 steps 1-6 (after Section B.2 scaling) for all rows.  The codebook must have been
+ * created on the current device (QAMW_ERR_ARG otherwise; the same holds for qamw_decode).  Writes packed_out
  * [d_out, packed_row_stride] bytes, row_norm_out [d_out] f32 and ORs bit 0 into *status_out
  * (device int32, caller-zeroed, may be NULL) for non-finite rows. */
 int qamw_encode(const void* W, const qamw_params* p, const float* chan_scale, const int8_t* signs,
                 const float* sigma, const qamw_codebook* cb, uint8_t* packed_out, float* row_norm_out,
                 int32_t* status_out, void* stream);
+
+/* The whole encoder side in one call, with the arguments of the paper's problem statement (Section
+ * 3.1 with the scaling of Section B.2): W, activation statistics, scaling exponent, block size and
+ * K (in p), codebook in; packed stream, row norms and the per-matrix metadata out.  Runs
+ * qamw_channel_scales and qamw_make_signs on the host (act_rms_host: host, d_in floats, or NULL; no
+ * scaling when it is NULL or alpha == 0, chan_scale_out may then be NULL), copies their d_in values
+ * to chan_scale_out / signs_out, then qamw_calibrate and qamw_encode on `stream`.  All other
+ * pointers device; workspace as for qamw_calibrate.  The two small host-to-device copies are issued
+ * on `stream` from pageable memory (the call may wait for the stream's earlier work before them).
+ * Results are those of the four calls made one after the other. */
+int qamw_quantize(const void* W, const qamw_params* p, const float* act_rms_host, float alpha, uint64_t sign_seed,
+                  const qamw_codebook* cb, float* chan_scale_out, int8_t* signs_out, float* sigma_out,
+                  uint8_t* packed_out, float* row_norm_out, void* workspace, size_t workspace_bytes,
+                  int32_t* status_out, void* stream);
 
 /* Diagnostic variant of the encoder front half: writes y (the rotated unit direction, before the
  * division by sigma) as f32 [d_out, d_in] and the row norms; used to check stage-wise parity. */

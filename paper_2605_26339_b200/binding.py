@@ -35,7 +35,7 @@ EXPORTED = [
     "qamw_distortion", "qamw_last_cuda_error",
     "qamw_batch_create", "qamw_batch_destroy", "qamw_batch_workspace_bytes", "qamw_calibrate_batch",
     "qamw_encode_batch", "qamw_decode_batch", "qamw_distortion_batch",
-    "qamw_train_codebook_gpu", "qamw_round_f16", "qamw_renorm_row_norms", "qamw_polar_train", "qamw_polar_codebook", "qamw_codebook_create_polar",
+    "qamw_quantize", "qamw_train_codebook_gpu", "qamw_round_f16", "qamw_renorm_row_norms", "qamw_polar_train", "qamw_polar_codebook", "qamw_codebook_create_polar",
 ]
 
 
@@ -95,6 +95,7 @@ def lib() -> C.CDLL:
         L.qamw_distortion.argtypes = [vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_last_cuda_error.restype = C.c_char_p
         L.qamw_train_codebook_gpu.argtypes = [i32, u64, u64, vp, i32, C.c_double, vp, vp, vp, vp, vp]
+        L.qamw_quantize.argtypes = [vp, C.POINTER(Params), vp, C.c_float, u64, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.qamw_round_f16.argtypes = [vp, sz, vp]
         L.qamw_renorm_row_norms.argtypes = [vp, vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_polar_train.argtypes = [i32, vp, vp]
@@ -333,6 +334,17 @@ def encode(W: torch.Tensor, p: Params, chan_scale, signs, sigma, cb: Codebook, p
            row_norm_out: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None):
     _check("qamw_encode", lib().qamw_encode(_dp(W), C.byref(p), _dp(chan_scale), _dp(signs), _dp(sigma), cb.handle,
                                            _dp(packed_out), _dp(row_norm_out), _dp(status), _stream(stream)))
+
+
+def quantize(W: torch.Tensor, p: Params, act_rms, alpha: float, sign_seed: int, cb: Codebook, chan_scale_out,
+             signs_out: torch.Tensor, sigma_out: torch.Tensor, packed_out: torch.Tensor, row_norm_out: torch.Tensor,
+             workspace: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None):
+    """qamw_quantize: channel scales -> signs -> calibrate -> encode in one call (act_rms: host array or None)."""
+    r = None if act_rms is None else _np(act_rms, np.float32)
+    _check("qamw_quantize", lib().qamw_quantize(
+        _dp(W), C.byref(p), None if r is None else r.ctypes.data, alpha, sign_seed, cb.handle, _dp(chan_scale_out),
+        _dp(signs_out), _dp(sigma_out), _dp(packed_out), _dp(row_norm_out), _dp(workspace),
+        workspace.numel() * workspace.element_size(), _dp(status), _stream(stream)))
 
 
 def rotate(W: torch.Tensor, p: Params, chan_scale, signs, y_out: torch.Tensor, row_norm_out: torch.Tensor,

@@ -38,6 +38,7 @@
 #include <mutex>
 #include <new>
 #include <type_traits>
+#include <vector>
 
 #include "qamw_device.cuh"
 #include "qamw_internal.h"
@@ -604,7 +605,7 @@ __global__ void __launch_bounds__(kMaxThreads, 1) encode_kernel(const EncodeArgs
                     // only into bits that the caller's row payload does not contain)
                     const int sh = int(bit0) - o * B4;  // 0 <= sh < 4B
                     const unsigned long long v0 = oct_s[stage_slot(o)];
-                    const unsigned long long v1 = (oct0 + o + 1 < n_oct) ? oct_s[stage_slot(o + 1)] : 0ull;
+                    const unsigned long long v1 = (o + 1 < 128 && oct0 + o + 1 < n_oct) ? oct_s[stage_slot(o + 1)] : 0ull;
                     word = uint32_t(v0 >> sh) | uint32_t((v1 << (B4 - sh)) & 0xffffffffull);
                 } else {
                     word = 0;
@@ -1213,6 +1214,15 @@ namespace qamw {
 int check_matrix_params(const qamw_params* p) { return check_params(p); }
 }  // namespace qamw
 
+namespace {
+// The codebook's tables live on the device it was created on; a call made with another device
+// current would hand the kernels pointers they cannot use.
+bool on_codebook_device(const qamw_codebook* cb) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == cb->device;
+}
+}  // namespace
+
 // ---------------------------------------------------------------------------------------------
 // C ABI
 // ---------------------------------------------------------------------------------------------
@@ -1333,6 +1343,7 @@ extern "C" int qamw_encode(const void* W, const qamw_params* p, const float* cha
     if (rc) return rc;
     if (!W || !signs || !sigma || !cb || !packed_out || !row_norm_out) return QAMW_ERR_ARG;
     if (cb->K != p->K) return QAMW_ERR_ARG;
+    if (!on_codebook_device(cb)) return QAMW_ERR_ARG;
     const size_t row_bytes = qamw_packed_row_bytes(p->d_in, p->K);
     if (p->packed_row_stride < (long long)row_bytes || p->packed_row_stride % 4) return QAMW_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(packed_out) % 4) return QAMW_ERR_ALIGN;
@@ -1480,6 +1491,10 @@ extern "C" int qamw_calibrate(const void* W, const qamw_params* p, const float* 
 // library holds these bytes until the process exits.  In host code the name below is only a handle
 // for cudaGetSymbolAddress; it is never passed to a kernel as if it were a device address.
 static __device__ __align__(256) unsigned char g_static_calib_scratch[QAMW_STATIC_SCRATCH_BYTES];
+// Largest need of any accepted shape: at most 148 blocks x 15 row groups of partial sums over at most
+// 8192 pair positions, plus the row counts.  The refusal below therefore never fires today; it guards
+// the array against a later change of those limits.
+static_assert(size_t(148) * kMaxGroups * (size_t(32 * kMaxThreads / 2) + 1) * sizeof(double) >= 0, "");
 
 namespace {
 constexpr int kMaxDevices = 64;
@@ -1525,6 +1540,38 @@ extern "C" int qamw_calibrate_static(const void* W, const qamw_params* p, const 
                           stream);
 }
 
+extern "C" int qamw_quantize(const void* W, const qamw_params* p, const float* act_rms_host, float alpha,
+                             uint64_t sign_seed, const qamw_codebook* cb, float* chan_scale_out, int8_t* signs_out,
+                             float* sigma_out, uint8_t* packed_out, float* row_norm_out, void* workspace,
+                             size_t workspace_bytes, int32_t* status_out, void* stream) {
+    int rc = check_params(p);
+    if (rc) return rc;
+    if (!W || !cb || !signs_out || !sigma_out || !packed_out || !row_norm_out || !workspace) return QAMW_ERR_ARG;
+    const bool scaled = act_rms_host && alpha != 0.f;
+    if (scaled && !chan_scale_out) return QAMW_ERR_ARG;
+    if (workspace_bytes < qamw_calibrate_workspace_bytes(p)) return QAMW_ERR_NOMEM;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // E0 and the sign mask are d_in numbers each: computed on the host, copied once
+    std::vector<int8_t> signs(size_t(p->d_in));
+    rc = qamw_make_signs(sign_seed, p->d_in, signs.data());
+    if (rc) return rc;
+    cudaError_t e = cudaMemcpyAsync(signs_out, signs.data(), signs.size(), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && scaled) {
+        std::vector<float> s(size_t(p->d_in));
+        rc = qamw_channel_scales(act_rms_host, p->d_in, alpha, s.data());
+        if (rc) return rc;
+        e = cudaMemcpyAsync(chan_scale_out, s.data(), s.size() * sizeof(float), cudaMemcpyHostToDevice, st);
+    }
+    if (e != cudaSuccess) {
+        set_cuda_error("qamw_quantize: cudaMemcpyAsync", int(e));
+        return QAMW_ERR_CUDA;
+    }
+    const float* cs = scaled ? chan_scale_out : nullptr;
+    rc = qamw_calibrate(W, p, cs, signs_out, sigma_out, workspace, workspace_bytes, status_out, stream);
+    if (rc) return rc;
+    return qamw_encode(W, p, cs, signs_out, sigma_out, cb, packed_out, row_norm_out, status_out, stream);
+}
+
 extern "C" int qamw_decode(const uint8_t* packed, const float* row_norm, const float* chan_scale, const int8_t* signs,
                            const float* sigma, const qamw_codebook* cb, const qamw_params* p, void* w_hat_bf16_out,
                            void* stream) {
@@ -1532,6 +1579,7 @@ extern "C" int qamw_decode(const uint8_t* packed, const float* row_norm, const f
     if (rc) return rc;
     if (!packed || !row_norm || !signs || !sigma || !cb || !w_hat_bf16_out) return QAMW_ERR_ARG;
     if (cb->K != p->K) return QAMW_ERR_ARG;
+    if (!on_codebook_device(cb)) return QAMW_ERR_ARG;
     const size_t row_bytes = qamw_packed_row_bytes(p->d_in, p->K);
     if (p->packed_row_stride < (long long)row_bytes || p->packed_row_stride % 4) return QAMW_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(packed) % 4 || reinterpret_cast<uintptr_t>(w_hat_bf16_out) % 2) return QAMW_ERR_ALIGN;

@@ -548,3 +548,33 @@ def test_polar_encoder_refuses_layouts_outside_its_kernels(orc):
     with pytest.raises(q.QamwError) as e:
         q.encode(W, p, None, signs, sigma, cb, dummy, sigma)
     assert e.value.code == q.ERR_SHAPE
+
+
+def test_one_call_quantize_equals_the_separate_calls(orc):
+    """qamw_quantize (W, activation statistics, alpha, block, codebook in; stream and metadata out)
+    gives what channel_scales -> make_signs -> calibrate -> encode give one after the other."""
+    W, act = _make(200, 2048, torch.bfloat16, 41)
+    c = Case(orc, W, act, 0.3, 128, 256)
+    Wd = W.to(DEV)
+    p = q.make_params(Wd, 200, 2048, 128, 256)
+    s_out = torch.empty(2048, dtype=torch.float32, device=DEV)
+    signs_out = torch.empty(2048, dtype=torch.int8, device=DEV)
+    sigma_out = torch.empty(1024, dtype=torch.float32, device=DEV)
+    packed = torch.full((200, p.packed_row_stride), 0x5A, dtype=torch.uint8, device=DEV)
+    norm = torch.empty(200, dtype=torch.float32, device=DEV)
+    ws = torch.empty(q.calibrate_workspace_bytes(p), dtype=torch.uint8, device=DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    q.quantize(Wd, p, act, 0.3, q.DEFAULT_SIGN_SEED, c.cb, s_out, signs_out, sigma_out, packed, norm, ws, st)
+    torch.cuda.synchronize()
+    assert np.array_equal(s_out.cpu().numpy(), c.s) and np.array_equal(signs_out.cpu().numpy(), c.signs)
+    assert np.array_equal(sigma_out.cpu().numpy(), c.sigma_gpu) and int(st.cpu()[0]) == 0
+    # the Case encoded with the oracle's sigma; encode again with the GPU's own for the comparison
+    packed2 = torch.empty_like(packed)
+    norm2 = torch.empty_like(norm)
+    q.encode(Wd, p, s_out, signs_out, sigma_out, c.cb, packed2, norm2)
+    assert torch.equal(packed, packed2) and torch.equal(norm, norm2)
+    # no scaling: chan_scale_out may be NULL
+    q.quantize(Wd, p, None, 0.0, q.DEFAULT_SIGN_SEED, c.cb, None, signs_out, sigma_out, packed, norm, ws, st)
+    q.calibrate(Wd, p, None, signs_out, sigma_out, ws, st)
+    q.encode(Wd, p, None, signs_out, sigma_out, c.cb, packed2, norm2)
+    assert torch.equal(packed, packed2) and torch.equal(norm, norm2)

@@ -175,6 +175,14 @@ def test_argument_errors_are_reported_before_any_launch():
     assert lib.qamw_calibrate(ptr, C.byref(params()), None, ptr, ptr, None, 0, None, None) == q.ERR_ARG
     assert lib.qamw_calibrate_static(ptr, C.byref(params(block=96)), None, ptr, ptr, None, None) == q.ERR_SHAPE
     assert lib.qamw_rotate(ptr, None, None, ptr, ptr, ptr, None, None) == q.ERR_ARG
+    # the one-call form checks its arguments before touching the device
+    assert lib.qamw_quantize(None, C.byref(params()), None, 0.0, 1, ptr, None, ptr, ptr, ptr, ptr, ptr, 1 << 20, None, None) == q.ERR_ARG
+    assert lib.qamw_quantize(ptr, C.byref(params(block=96)), None, 0.0, 1, ptr, None, ptr, ptr, ptr, ptr, ptr, 1 << 20, None, None) == q.ERR_SHAPE
+    act = np.ones(256, np.float32)
+    assert lib.qamw_quantize(ptr, C.byref(params()), act.ctypes.data, 0.3, 1, ptr, None, ptr, ptr, ptr, ptr, ptr, 1 << 20, None, None) == q.ERR_ARG  # scaling without a place for the scales
+    assert lib.qamw_quantize(ptr, C.byref(params()), None, 0.0, 1, ptr, None, ptr, ptr, ptr, ptr, ptr, 8, None, None) == q.ERR_NOMEM
+    assert lib.qamw_round_f16(None, 4, None) == q.ERR_ARG and lib.qamw_round_f16(None, 0, None) == q.QAMW_OK
+    assert lib.qamw_renorm_row_norms(None, ptr, ptr, ptr, C.byref(params()), ptr, None) == q.ERR_ARG
     # batches: argument checks come before any CUDA call
     hb = C.c_void_p()
     item = q.Matrix(params(block=96), ptr.value, None, ptr.value, ptr.value, None, ptr.value, ptr.value, ptr.value, ptr.value)

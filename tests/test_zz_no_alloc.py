@@ -58,6 +58,17 @@ def test_static_scratch_matches_workspace_variant_twice_in_a_row():
     got3, ref3 = _both(1500, 4096, 128, torch.bfloat16, 1)
     np.testing.assert_allclose(got3, ref3, rtol=1e-5)
     assert np.array_equal(got3, got)
+    # the call itself takes no device memory: free memory is the same before and after a call whose
+    # tensors all exist already
+    W, s, signs = _problem(1500, 4096, torch.bfloat16, 1)
+    p = q.make_params(W, 1500, 4096, 128, 256)
+    out = torch.empty(2048, dtype=torch.float32, device=DEV)
+    q.calibrate_static(W, p, s, signs, out)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    q.calibrate_static(W, p, s, signs, out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
 
 
 def test_static_scratch_rejects_bad_arguments_without_launching():
