@@ -91,6 +91,9 @@ struct MatDesc {
     double* dist4;
     long long w_row_stride;       // elements
     long long packed_row_stride;  // bytes
+    long long calib_offset;       // batched calibration: byte offset of this matrix's partial sums in the workspace,
+    int calib_first_block;        //   the first block whose span touches it, and the number of slots it has
+    int calib_slots;              //   ((blocks touching it) x (row groups per block)), each [pair_stride] doubles
     int d_out, d_in;
 };
 
@@ -100,9 +103,13 @@ struct MatDesc {
 int rows_decode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, const void* spans_dev, int span_blocks,
                 int block, int K, const float* codebook_dev, uint32_t flags, void* stream);
 int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, const void* spans_dev, int span_blocks,
-                int block, int K, int w_bf16, const ::qamw_codebook* cb, uint32_t flags, int32_t* status, void* stream);
+                int block, int K, int w_bf16, const ::qamw_codebook* cb, uint32_t flags, int32_t* status, void* stream,
+                void* calib_base = nullptr);  // calib_base: run the calibration pass instead (cb may be NULL)
 int sm_count();
-int check_matrix_params(const qamw_params* p);  // QAMW_OK or the error code every entry point reports
+int check_matrix_params(const qamw_params* p);
+long long distortion_items(int d_out, int d_in);  // work items of the distortion kernel for one matrix
+// zeroes every matrix's four sums, then one launch over all matrices (spans of the concatenated item list)
+int distortion_batch_launch(const MatDesc* descs_dev, int n, const void* spans_dev, int blocks, int w_bf16, void* stream);  // QAMW_OK or the error code every entry point reports
 
 }  // namespace qamw
 

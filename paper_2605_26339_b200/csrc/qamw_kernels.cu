@@ -996,15 +996,19 @@ __device__ __forceinline__ void dist_load(const void* W, long long w_row_stride,
     }
 }
 
+__host__ __device__ inline long long dist_item_count(int d_out, int d_in) {
+    return (long long)((d_in + 8 * kDistThreads - 1) / (8 * kDistThreads)) * ((d_out + kDistRows - 1) / kDistRows);
+}
+
+// The work items `first`, `first + step`, ... below `last` of one matrix, added into the thread's
+// four running sums.
 template <bool BF16>
-__global__ void __launch_bounds__(kDistThreads, 5) distortion_kernel(const void* W, long long w_row_stride,
-                                                                  const __nv_bfloat16* What, const float* act_rms,
-                                                                  int d_out, int d_in, int vec, double* out4) {
+__device__ __forceinline__ void dist_items(const void* W, long long w_row_stride, const __nv_bfloat16* What,
+                                           const float* act_rms, int d_out, int d_in, int vec, long long first,
+                                           long long last, long long step, double& s0, double& s1, double& s2,
+                                           double& s3) {
     const int col_tiles = (d_in + 8 * kDistThreads - 1) / (8 * kDistThreads);
-    const int row_chunks = (d_out + kDistRows - 1) / kDistRows;
-    const long long n_items = (long long)col_tiles * row_chunks;
-    double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
-    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+    for (long long item = first; item < last; item += step) {
         const int chunk = int(item / col_tiles), tile = int(item - (long long)chunk * col_tiles);
         const int j0 = (tile * kDistThreads + threadIdx.x) * 8;
         if (j0 >= d_in) continue;
@@ -1089,9 +1093,14 @@ __global__ void __launch_bounds__(kDistThreads, 5) distortion_kernel(const void*
             s3 = fma(r2, Q[e], s3);
         }
     }
+}
+
+// Block-wide sums of the four values (fixed order inside the block), added to out4 by four threads.
+__device__ __forceinline__ void dist_flush(double s0, double s1, double s2, double s3, double* out4) {
     __shared__ double sh[4][kDistThreads / 32];
     s0 = warp_sum(s0); s1 = warp_sum(s1); s2 = warp_sum(s2); s3 = warp_sum(s3);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();  // a previous flush has been read
     if (lane == 0) { sh[0][warp] = s0; sh[1][warp] = s1; sh[2][warp] = s2; sh[3][warp] = s3; }
     __syncthreads();
     if (threadIdx.x < 4) {
@@ -1099,6 +1108,40 @@ __global__ void __launch_bounds__(kDistThreads, 5) distortion_kernel(const void*
         for (int w = 0; w < kDistThreads / 32; ++w) v += sh[threadIdx.x][w];
         atomicAdd(out4 + threadIdx.x, v);
     }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kDistThreads, 5) distortion_kernel(const void* W, long long w_row_stride,
+                                                                  const __nv_bfloat16* What, const float* act_rms,
+                                                                  int d_out, int d_in, int vec, double* out4) {
+    const long long n_items = dist_item_count(d_out, d_in);
+    double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+    dist_items<BF16>(W, w_row_stride, What, act_rms, d_out, d_in, vec, blockIdx.x, n_items, gridDim.x, s0, s1, s2, s3);
+    dist_flush(s0, s1, s2, s3, out4);
+}
+
+// All matrices of a batch: block b owns a contiguous span of the concatenated item list.
+template <bool BF16>
+__global__ void __launch_bounds__(kDistThreads, 5) distortion_batch_kernel(const MatDesc* descs, const int4* spans) {
+    const int4 span = spans[blockIdx.x];
+    for (int m = span.x; m <= span.z; ++m) {
+        const MatDesc& d = descs[m];
+        const long long first = m == span.x ? span.y : 0;
+        const long long last = m == span.z ? span.w : dist_item_count(d.d_out, d.d_in);
+        if (first >= last) continue;
+        const size_t esz = BF16 ? 2 : 4;
+        const int vec = (d.d_in % 8 == 0) && (reinterpret_cast<uintptr_t>(d.W) % 16 == 0) &&
+                        ((size_t(d.w_row_stride) * esz) % 16 == 0) && (reinterpret_cast<uintptr_t>(d.w_hat) % 16 == 0);
+        double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+        dist_items<BF16>(d.W, d.w_row_stride, static_cast<const __nv_bfloat16*>(d.w_hat), d.act_rms, d.d_out, d.d_in, vec,
+                         first, last, 1, s0, s1, s2, s3);
+        dist_flush(s0, s1, s2, s3, d.dist4);
+    }
+}
+
+__global__ void zero_dist_kernel(const MatDesc* descs, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < 4 * n) descs[i >> 2].dist4[i & 3] = 0.0;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1212,6 +1255,14 @@ int launch_decode(const DecodeArgs& a, int blocks, size_t smem, cudaStream_t st)
 
 namespace qamw {
 int check_matrix_params(const qamw_params* p) { return check_params(p); }
+long long distortion_items(int d_out, int d_in) { return dist_item_count(d_out, d_in); }
+int distortion_batch_launch(const MatDesc* descs_dev, int n, const void* spans_dev, int blocks, int w_bf16, void* stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    zero_dist_kernel<<<(4 * n + 255) / 256, 256, 0, st>>>(descs_dev, n);
+    if (w_bf16) distortion_batch_kernel<true><<<blocks, kDistThreads, 0, st>>>(descs_dev, static_cast<const int4*>(spans_dev));
+    else distortion_batch_kernel<false><<<blocks, kDistThreads, 0, st>>>(descs_dev, static_cast<const int4*>(spans_dev));
+    return finish_launch("distortion_batch_kernel");
+}
 }  // namespace qamw
 
 namespace {

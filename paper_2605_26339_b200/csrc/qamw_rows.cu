@@ -394,6 +394,7 @@ struct Encode2Args {
     int brute;
     float inv_sqrt_b;        // c_b = f32(1 / sqrt(b))
     int32_t* status;         // out (optional): bit 0 set when a row norm is not finite
+    unsigned char* calib_base;  // calibration mode: base of the partial-sum workspace (MatDesc::calib_offset)
     int polar_ba, polar_bp;  // polar quantiser: amplitude and phase bits; `table` then holds the squared
                              // amplitude thresholds (2^Ba floats) and, from off_overflow on, the unit vectors
                              // of the phase bin boundaries of the upper half plane (2^Bp / 2 float2)
@@ -446,8 +447,14 @@ struct Stage2 {
 // adds up its part of the row norm, rotates (shuffles only), and after the one meeting point of the
 // row's warps -- a named barrier for the norm -- searches its 256 pairs, stages the indices and
 // writes its 32 B bytes of the packed row.  W is read once.
-template <bool BF16, int LOG2B, int NS, int MAXT, bool POLAR>
+// QUANT: 0 = nearest codeword through the cell table, 1 = polar quantiser, 2 = no quantiser at all:
+// the kernel then is the calibration pass of Section 3.4, which visits n = min(d_out, 1024) rows
+// floor(t d_out / n) and adds up the pair moduli |(y_2k, y_2k+1)| per pair position.  Every row group
+// of every block owns one slot of partial sums in the workspace; calibrate_finish2_kernel adds the
+// slots in ascending order, so the result does not depend on timing.
+template <bool BF16, int LOG2B, int NS, int MAXT, int QUANT>
 __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
+    constexpr bool POLAR = QUANT == 1, CALIB = QUANT == 2;
     constexpr int WE = 256 * NS;
     typedef Lay2<NS, LOG2B> Lay;
     extern __shared__ __align__(16) unsigned char smem[];
@@ -455,10 +462,10 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
     __shared__ MatDesc cur;            // the matrix the block is working on (re-read per row: saves registers)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
 
-    const int cb_bytes = POLAR ? 0 : (a.K * 8) << a.log2c;  // the polar quantiser never reads codewords
-    if (!POLAR) fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
+    const int cb_bytes = QUANT != 0 ? 0 : (a.K * 8) << a.log2c;  // only the table search reads codewords
+    if (QUANT == 0) fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c);
     unsigned char* table = smem + cb_bytes;
-    {
+    if (!CALIB) {
         uint4* dst = reinterpret_cast<uint4*>(table);
         const int n16 = a.table_bytes / 16;
         for (int base = 0; base < n16; base += 8 * blockDim.x) {
@@ -511,7 +518,8 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
         const MatDesc& d = cur;
         const int d_in = d.d_in, n_pairs = d_in >> 1;
         const int row_begin = m == span.x ? span.y : 0;
-        const int row_end = m == span.z ? span.w : d.d_out;
+        const int n_cal = min(d.d_out, QAMW_CALIB_MAX_ROWS);  // calibration walks this many rows
+        const int row_end = m == span.z ? span.w : (CALIB ? n_cal : d.d_out);
         const int n_seg = (d_in + WE - 1) / WE;
         const int groups = min(15, n_warps / n_seg);  // named barriers 1..15
         const int group = warp / n_seg, seg = warp - group * n_seg;
@@ -542,7 +550,12 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
             for (int i = 0; i < 4; ++i) t[p][i] = pack2(cs[2 * i] * sgn[2 * i], cs[2 * i + 1] * sgn[2 * i + 1]);
             const int k0 = 4 * (oct0 + Lay::octet_after(lane, p));
             live[p] = k0 < n_pairs;
-            load4f(d.sigma, k0, n_pairs, 1, 1.0f, q[p]);
+            if (!CALIB) {
+                load4f(d.sigma, k0, n_pairs, 1, 1.0f, q[p]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) q[p][i] = 1.0f;
+            }
             const float fl = Lay::negated(lane, p) ? -1.0f : 1.0f;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -563,14 +576,21 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
         double* part_base = &ss_part[0][group * n_seg];
 
         auto rows = [&](auto mode_tag) {
-            constexpr int MODE = decltype(mode_tag)::value;  // 0 = table, 1 = table with reach check, 2 = exhaustive, 3 = polar
+            constexpr int MODE = decltype(mode_tag)::value;  // 0 = table, 1 = table with reach check, 2 = exhaustive, 3 = polar, 4 = calibrate
             int parity = 0;
+            double acc[NS][4];
+            int used = 0;
+#pragma unroll
+            for (int p = 0; p < NS; ++p)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[p][i] = 0.0;
             // raw bits of the thread's elements of one row; the next row is fetched as soon as this one
             // has been converted, so its latency hides behind the rotation and the search
             constexpr int kRaw = BF16 ? 4 * NS : 8 * NS;
             uint32_t raw[kRaw];
-            auto fetch = [&](int row) {
-                const char* wp = static_cast<const char*>(cur.W) + ((long long)row * cur.w_row_stride + col0) * kEsz;
+            auto fetch = [&](int t) {
+                const long long row = CALIB ? (long long)t * cur.d_out / n_cal : t;
+                const char* wp = static_cast<const char*>(cur.W) + (row * cur.w_row_stride + col0) * kEsz;
 #pragma unroll
                 for (int h = 0; h < kRaw / 8; ++h) {
                     uint32_t w[8];
@@ -625,12 +645,25 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
                     // row (its indices are unspecified; the searches accept any input)
                     if (isfinite(r) && r > 0.f) gn = __fdiv_rn(a.inv_sqrt_b, r);
                     if (seg == 0) {
-                        cur.row_norm[row] = r;
+                        if (!CALIB) cur.row_norm[row] = r;
                         if (!isfinite(r) && a.status) atomicOr(a.status, 1);
                     }
                 }
                 gn = __shfl_sync(kFull, gn, 0);
                 const f32x2 gn2 = pack2(gn, gn);
+                if constexpr (MODE == 4) {  // calibration: rows of zero (or non-finite) norm are skipped
+                    if (gn != 0.f) {
+                        ++used;
+#pragma unroll
+                        for (int p = 0; p < NS; ++p)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                float y0, y1;
+                                unpack2(mul2(P[p][i], gn2), y0, y1);
+                                acc[p][i] += double(sqrtf(__fmaf_rn(y1, y1, __fmul_rn(y0, y0))));
+                            }
+                    }
+                } else {
 #pragma unroll
                 for (int p = 0; p < NS; ++p) {
                     uint32_t v[4];
@@ -697,9 +730,26 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
                 if (last_seg)  // padding up to the row stride is written as zero
                     for (int gw = payload_words + lane; gw < row_words; gw += 32) out[gw] = 0u;
                 __syncwarp();  // the staging piece is free again
+                }  // MODE != 4
+            }
+            if constexpr (MODE == 4) {  // this row group's sums go to its own slot of the matrix's workspace
+                const int pair_stride = (n_pairs + 3) & ~3;
+                const int slot = (int(blockIdx.x) - cur.calib_first_block) * groups + group;
+                double* ws = reinterpret_cast<double*>(a.calib_base + cur.calib_offset);
+                double* mine = ws + size_t(slot) * pair_stride;
+#pragma unroll
+                for (int p = 0; p < NS; ++p)
+                    if (live[p]) {
+                        const int k0 = 4 * (oct0 + Lay::octet_after(lane, p));
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) mine[k0 + i] = acc[p][i];
+                    }
+                if (lane == 0 && seg == 0) ws[size_t(cur.calib_slots) * pair_stride + slot] = double(used);
             }
         };
-        if constexpr (POLAR) {
+        if constexpr (CALIB) {
+            rows(std::integral_constant<int, 4>{});
+        } else if constexpr (POLAR) {
             rows(std::integral_constant<int, 3>{});
         } else {
             if (a.brute) rows(std::integral_constant<int, 2>{});
@@ -707,6 +757,25 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
             else rows(std::integral_constant<int, 0>{});
         }
     }
+}
+
+// sigma_k of every matrix from the slots of partial sums (zeroed before the calibration pass, so a
+// slot nobody wrote counts as empty): thread = one pair position, slots added in ascending order.
+__global__ void calibrate_finish2_kernel(const MatDesc* descs, const unsigned char* calib_base) {
+    const MatDesc& d = descs[blockIdx.y];
+    const int n_pairs = d.d_in >> 1, pair_stride = (n_pairs + 3) & ~3;
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= n_pairs) return;
+    const double* ws = reinterpret_cast<const double*>(calib_base + d.calib_offset);
+    double s = 0.0, u = 0.0;
+    for (int slot = 0; slot < d.calib_slots; ++slot) {
+        s += ws[size_t(slot) * pair_stride + k];
+        u += ws[size_t(d.calib_slots) * pair_stride + slot];
+    }
+    const double inv_sqrt_d = 1.0 / sqrt(double(d.d_in));
+    double sg = u > 0.0 ? (s / u) / sqrt(1.5707963267948966) : inv_sqrt_d;  // Rayleigh mean = sigma sqrt(pi / 2)
+    sg = fmax(sg, 1e-4 * inv_sqrt_d);
+    const_cast<float*>(d.sigma)[k] = float(sg);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -761,15 +830,21 @@ int launch_decode2(const Decode2Args& a, int blocks, int threads, size_t smem, c
 
 template <bool BF16, int LOG2B, int NS, int MAXT>
 int launch_encode2(const Encode2Args& a, int blocks, int threads, size_t smem, cudaStream_t st) {
-    if (a.polar_ba >= 0) {
-        int rc = raise_smem_limit(reinterpret_cast<const void*>(&encode2_kernel<BF16, LOG2B, NS, MAXT, true>));
+    if (a.calib_base) {
+        int rc = raise_smem_limit(reinterpret_cast<const void*>(&encode2_kernel<BF16, LOG2B, NS, MAXT, 2>));
         if (rc) return rc;
-        encode2_kernel<BF16, LOG2B, NS, MAXT, true><<<blocks, threads, smem, st>>>(a);
+        encode2_kernel<BF16, LOG2B, NS, MAXT, 2><<<blocks, threads, smem, st>>>(a);
+        return launch_check("encode2_kernel (calibrate)");
+    }
+    if (a.polar_ba >= 0) {
+        int rc = raise_smem_limit(reinterpret_cast<const void*>(&encode2_kernel<BF16, LOG2B, NS, MAXT, 1>));
+        if (rc) return rc;
+        encode2_kernel<BF16, LOG2B, NS, MAXT, 1><<<blocks, threads, smem, st>>>(a);
         return launch_check("encode2_kernel (polar)");
     }
-    int rc = raise_smem_limit(reinterpret_cast<const void*>(&encode2_kernel<BF16, LOG2B, NS, MAXT, false>));
+    int rc = raise_smem_limit(reinterpret_cast<const void*>(&encode2_kernel<BF16, LOG2B, NS, MAXT, 0>));
     if (rc) return rc;
-    encode2_kernel<BF16, LOG2B, NS, MAXT, false><<<blocks, threads, smem, st>>>(a);
+    encode2_kernel<BF16, LOG2B, NS, MAXT, 0><<<blocks, threads, smem, st>>>(a);
     return launch_check("encode2_kernel");
 }
 
@@ -874,7 +949,8 @@ int decode_groups(int n_seg) { return 16 / n_seg; }
 constexpr int kCostUnit = 360360;  // divisible by every group count 1..15
 
 int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, const void* spans_dev, int span_blocks,
-                int block, int K, int w_bf16, const ::qamw_codebook* cb, uint32_t flags, int32_t* status, void* stream) {
+                int block, int K, int w_bf16, const ::qamw_codebook* cb, uint32_t flags, int32_t* status, void* stream,
+                void* calib_base) {
     constexpr int NS = 2, WE = 256 * NS;
     const int log2b = ilog2(block);
     if (log2b < 5 || log2b > 9 || n <= 0) return QAMW_ERR_SHAPE;
@@ -885,7 +961,7 @@ int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, cons
         const MatDesc& d = descs_host[i];
         if (d.d_in % (8 * NS)) return QAMW_ERR_SHAPE;
         if (!aligned(d.W, 32) || (size_t(d.w_row_stride) * esz) % 32) return QAMW_ERR_SHAPE;
-        if (!aligned(d.chan_scale, 16) || !aligned(d.signs, 8) || !aligned(d.sigma, 16)) return QAMW_ERR_SHAPE;
+        if (!aligned(d.chan_scale, 16) || !aligned(d.signs, 8) || (!calib_base && !aligned(d.sigma, 16))) return QAMW_ERR_SHAPE;
         const int n_seg = (d.d_in + WE - 1) / WE;
         max_seg = std::max(max_seg, n_seg);
         warps = std::max(warps, encode_warps(n_seg));
@@ -897,27 +973,31 @@ int rows_encode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, cons
     a.descs = descs_dev;
     a.one = descs_host[0];
     a.spans = static_cast<const int4*>(spans_dev);
-    a.codebook = static_cast<const float2*>(cb->d_blob);
-    a.table = reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(cb->d_blob) + cb->off_cells);
-    a.table_bytes = int(cb->blob_bytes - cb->off_cells);
-    a.off_overflow = int(cb->off_overflow - cb->off_cells);
+    a.calib_base = static_cast<unsigned char*>(calib_base);
+    const bool calib = calib_base != nullptr;
+    a.codebook = calib ? nullptr : static_cast<const float2*>(cb->d_blob);
+    a.table = calib ? nullptr : reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(cb->d_blob) + cb->off_cells);
+    a.table_bytes = calib ? 0 : int(cb->blob_bytes - cb->off_cells);
+    a.off_overflow = calib ? 0 : int(cb->off_overflow - cb->off_cells);
     a.K = K;
     a.log2K = ilog2(K);
-    a.grid = cb->map.grid;
-    a.map_zmax = cb->map.zmax;
-    a.map_c0 = cb->map.c0;
-    a.map_c1 = cb->map.c1;
-    a.map_c2 = cb->map.c2;
-    a.map_bias = 12582912.0f + float(cb->map.half);
+    a.grid = calib ? 1 : cb->map.grid;
+    a.map_zmax = calib ? 0.f : cb->map.zmax;
+    a.map_c0 = calib ? 0.f : cb->map.c0;
+    a.map_c1 = calib ? 0.f : cb->map.c1;
+    a.map_c2 = calib ? 0.f : cb->map.c2;
+    a.map_bias = calib ? 0.f : 12582912.0f + float(cb->map.half);
     a.brute = (flags & QAMW_FLAG_BRUTE_FORCE) ? 1 : 0;
     a.inv_sqrt_b = float(1.0 / std::sqrt(double(block)));
     a.status = status;
-    a.polar_ba = cb->polar ? cb->polar_ba : -1;
-    a.polar_bp = cb->polar ? cb->polar_bp : -1;
+    const bool polar = !calib && cb->polar;
+    a.polar_ba = polar ? cb->polar_ba : -1;
+    a.polar_bp = polar ? cb->polar_bp : -1;
     const size_t fixed = ((size_t(a.table_bytes) + 15) & ~size_t(15)) + size_t(warps) * Stage2<NS>::kSlots * 8;
-    if (fixed + size_t(K) * 8 > kSmemLimit - kEncode2StaticSmem) return QAMW_ERR_SHAPE;
-    a.log2c = cb->polar ? 0 : pick_copies(K, kSmemLimit - kEncode2StaticSmem - fixed);
-    const size_t smem = fixed + (cb->polar ? 0 : (size_t(K) * 8 << a.log2c));
+    if (!calib && fixed + size_t(K) * 8 > kSmemLimit - kEncode2StaticSmem) return QAMW_ERR_SHAPE;
+    const bool tables = !calib && !polar;
+    a.log2c = tables ? pick_copies(K, kSmemLimit - kEncode2StaticSmem - fixed) : 0;
+    const size_t smem = fixed + (tables ? (size_t(K) * 8 << a.log2c) : 0);
     int grid = sm_count();
     if (flags & QAMW_FLAG_HALF_DEVICE) grid = std::max(1, grid / 2);
     const int blocks = spans_dev ? span_blocks : int(std::max<long long>(1, std::min<long long>(grid, rows)));
@@ -970,6 +1050,10 @@ struct qamw_batch {
     int n_blocks = 0;
     RowSet dec;                     // all matrices, spans weighted for the decoder's geometry
     RowSet enc[3];                  // encoder: one set per block size (20, 24, 28 warps)
+    int4* d_spans_dist = nullptr;   // distortion: spans of the concatenated work-item list, over dec.d_descs
+    int n_blocks_dist = 0;
+    RowSet cal[3];                  // calibration: the encoder's sets again, spans over the calibration rows
+    size_t cal_bytes = 0;           // partial-sum slots of all matrices (front of the caller's workspace)
     std::vector<size_t> ws_offset;  // calibration scratch of item i inside the caller's workspace
     size_t ws_bytes = 0;
 };
@@ -1060,6 +1144,50 @@ extern "C" int qamw_batch_create(const qamw_matrix* items, int n, const qamw_cod
     }
     e = upload_row_set(b->dec, b->n_blocks, dec_cost);
     for (int c = 0; c < 3 && e == cudaSuccess; ++c) e = upload_row_set(b->enc[c], b->n_blocks, enc_cost[c]);
+    for (int c = 0; c < 3 && e == cudaSuccess; ++c) {  // calibration: min(d_out, 1024) rows per matrix
+        RowSet& r = b->cal[c];
+        r.index = b->enc[c].index;
+        r.descs = b->enc[c].descs;
+        if (r.descs.empty()) continue;
+        const int m = int(r.descs.size());
+        std::vector<MatDesc> cal_rows(r.descs);
+        for (MatDesc& d : cal_rows) d.d_out = std::min(d.d_out, QAMW_CALIB_MAX_ROWS);
+        std::vector<int4> spans;
+        make_spans(cal_rows.data(), m, b->n_blocks, enc_cost[c].data(), &spans);
+        std::vector<int> first(size_t(m), b->n_blocks), last(size_t(m), -1);
+        for (int k = 0; k < b->n_blocks; ++k)
+            for (int i = spans[size_t(k)].x; i <= spans[size_t(k)].z; ++i) {
+                first[size_t(i)] = std::min(first[size_t(i)], k);
+                last[size_t(i)] = std::max(last[size_t(i)], k);
+            }
+        for (int i = 0; i < m; ++i) {
+            MatDesc& d = r.descs[size_t(i)];
+            const int groups = kCostUnit / enc_cost[c][size_t(i)];
+            d.calib_first_block = first[size_t(i)];
+            d.calib_slots = std::max(0, last[size_t(i)] - first[size_t(i)] + 1) * groups;
+            d.calib_offset = (long long)b->cal_bytes;
+            const size_t pair_stride = (size_t(d.d_in / 2) + 3) & ~size_t(3);
+            b->cal_bytes += ((size_t(d.calib_slots) * (pair_stride + 1)) * sizeof(double) + 255) & ~size_t(255);
+        }
+        e = cudaMalloc(&r.d_descs, sizeof(MatDesc) * size_t(m));
+        if (e == cudaSuccess) e = cudaMemcpy(r.d_descs, r.descs.data(), sizeof(MatDesc) * size_t(m), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMalloc(&r.d_spans, sizeof(int4) * spans.size());
+        if (e == cudaSuccess) e = cudaMemcpy(r.d_spans, spans.data(), sizeof(int4) * spans.size(), cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess) {  // distortion: equal numbers of work items per block, sixteen blocks per SM
+        std::vector<MatDesc> items_as_rows(b->dec.descs);
+        std::vector<int> unit(size_t(n), 1);
+        long long total = 0;
+        for (int i = 0; i < n; ++i) {
+            items_as_rows[size_t(i)].d_out = int(distortion_items(b->dec.descs[size_t(i)].d_out, b->dec.descs[size_t(i)].d_in));
+            total += items_as_rows[size_t(i)].d_out;
+        }
+        b->n_blocks_dist = int(std::max<long long>(1, std::min<long long>(16LL * b->n_blocks, total)));
+        std::vector<int4> spans;
+        make_spans(items_as_rows.data(), n, b->n_blocks_dist, unit.data(), &spans);
+        e = cudaMalloc(&b->d_spans_dist, sizeof(int4) * spans.size());
+        if (e == cudaSuccess) e = cudaMemcpy(b->d_spans_dist, spans.data(), sizeof(int4) * spans.size(), cudaMemcpyHostToDevice);
+    }
     if (e != cudaSuccess) {
         set_cuda_error("qamw_batch_create", int(e));
         qamw_batch_destroy(b);
@@ -1072,24 +1200,61 @@ extern "C" int qamw_batch_create(const qamw_matrix* items, int n, const qamw_cod
 extern "C" void qamw_batch_destroy(qamw_batch* b) {
     if (!b) return;
     free_row_set(b->dec);
-    for (int c = 0; c < 3; ++c) free_row_set(b->enc[c]);
+    for (int c = 0; c < 3; ++c) {
+        free_row_set(b->enc[c]);
+        free_row_set(b->cal[c]);
+    }
+    if (b->d_spans_dist) cudaFree(b->d_spans_dist);
     delete b;
 }
 
-extern "C" size_t qamw_batch_workspace_bytes(const qamw_batch* b) { return b ? b->ws_bytes : 0; }
+// The front of the workspace holds the slots of the batched pass, the rest the scratch of the
+// single-matrix calls that matrices outside the common layout fall back to.
+extern "C" size_t qamw_batch_workspace_bytes(const qamw_batch* b) { return b ? b->cal_bytes + b->ws_bytes : 0; }
 
 extern "C" int qamw_calibrate_batch(const qamw_batch* b, void* workspace, size_t workspace_bytes, int32_t* status_out,
                                     void* stream) {
     if (!b || !workspace) return QAMW_ERR_ARG;
     if (reinterpret_cast<uintptr_t>(workspace) % 8) return QAMW_ERR_ALIGN;
-    if (workspace_bytes < b->ws_bytes) return QAMW_ERR_NOMEM;
+    if (workspace_bytes < b->cal_bytes + b->ws_bytes) return QAMW_ERR_NOMEM;
     for (int i = 0; i < b->n; ++i)
         if (!b->items[i].W || !b->items[i].sigma) return QAMW_ERR_ARG;
-    for (int i = 0; i < b->n; ++i) {
-        const qamw_matrix& it = b->items[i];
-        int rc = qamw_calibrate(it.W, &it.p, it.chan_scale, it.signs, it.sigma,
-                                static_cast<unsigned char*>(workspace) + b->ws_offset[i],
-                                workspace_bytes - b->ws_offset[i], status_out, stream);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t flags = b->items[0].p.flags;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    bool zeroed = false;
+    for (int c = 0; c < 3; ++c) {  // one pass and one finish launch per block size
+        const RowSet& set = b->cal[c];
+        if (set.descs.empty()) continue;
+        int rc = QAMW_ERR_SHAPE;
+        if (!(flags & QAMW_FLAG_GENERAL_KERNELS)) {
+            if (!zeroed) {  // a slot that no row group writes must read as empty
+                cudaError_t e = cudaMemsetAsync(ws, 0, b->cal_bytes, st);
+                if (e != cudaSuccess) {
+                    set_cuda_error("cudaMemsetAsync", int(e));
+                    return QAMW_ERR_CUDA;
+                }
+                zeroed = true;
+            }
+            rc = rows_encode(set.d_descs, set.descs.data(), int(set.descs.size()), set.d_spans, b->n_blocks, b->block, b->K,
+                             b->w_dtype == QAMW_DTYPE_BF16, nullptr, flags, status_out, stream, ws);
+            if (rc == QAMW_OK) {
+                int max_pairs = 0;
+                for (const MatDesc& d : set.descs) max_pairs = std::max(max_pairs, d.d_in / 2);
+                calibrate_finish2_kernel<<<dim3(unsigned((max_pairs + 255) / 256), unsigned(set.descs.size())), 256, 0, st>>>(
+                    set.d_descs, ws);
+                rc = launch_check("calibrate_finish2_kernel");
+            }
+        }
+        if (rc == QAMW_ERR_SHAPE) {  // some matrix of the set needs the general kernel: one call per matrix
+            rc = QAMW_OK;
+            for (size_t k = 0; k < set.index.size() && rc == QAMW_OK; ++k) {
+                const int i = set.index[k];
+                const qamw_matrix& it = b->items[i];
+                rc = qamw_calibrate(it.W, &it.p, it.chan_scale, it.signs, it.sigma, ws + b->cal_bytes + b->ws_offset[i],
+                                    workspace_bytes - b->cal_bytes - b->ws_offset[i], status_out, stream);
+            }
+        }
         if (rc) return rc;
     }
     return QAMW_OK;
@@ -1148,10 +1313,6 @@ extern "C" int qamw_distortion_batch(const qamw_batch* b, void* stream) {
         const qamw_matrix& it = b->items[i];
         if (!it.W || !it.w_hat_bf16 || !it.dist4) return QAMW_ERR_ARG;
     }
-    for (int i = 0; i < b->n; ++i) {
-        const qamw_matrix& it = b->items[i];
-        int rc = qamw_distortion(it.W, it.w_hat_bf16, it.act_rms, &it.p, it.dist4, stream);
-        if (rc) return rc;
-    }
-    return QAMW_OK;
+    return distortion_batch_launch(b->dec.d_descs, b->n, b->d_spans_dist, b->n_blocks_dist, b->w_dtype == QAMW_DTYPE_BF16,
+                                   stream);
 }

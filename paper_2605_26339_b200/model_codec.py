@@ -1,8 +1,8 @@
 """Whole-model driver over the C ABI: calibrate -> encode -> decode -> distortion for every
 linear weight of a (synthetic) checkpoint.  This is the call a user of the library makes to
-quantise a model.  Encode and decode go through one qamw_batch (a persistent launch per phase
-that walks all matrices); calibration and distortion are one library call per matrix, dealt
-onto a few side streams.
+quantise a model.  All four phases go through one qamw_batch: a persistent launch per phase (per
+class of row lengths for the encoder side) that walks all matrices.  With ``use_batch = False`` every
+phase is one library call per matrix, dealt onto a few side streams.
 """
 from __future__ import annotations
 
@@ -98,6 +98,7 @@ class ModelCodec:
     workspace: Optional[torch.Tensor] = None
     status: Optional[torch.Tensor] = None
     batch: Optional[q.Batch] = None
+    batch_workspace: Optional[torch.Tensor] = None
     use_batch: bool = True
     _meta_cache: Dict[int, Tuple[torch.Tensor, torch.Tensor]] = field(default_factory=dict)
 
@@ -125,6 +126,8 @@ class ModelCodec:
             mats = [q.make_matrix(s.params, s.W, s.chan_scale, s.signs, s.sigma, s.act_rms, s.packed, s.row_norm,
                                   s.w_hat, s.dist) for s in self.slots]
             self.batch = q.Batch(mats, self.codebook) if mats else None
+            self.batch_workspace = (torch.empty(max(8, self.batch.workspace_bytes()), dtype=torch.uint8, device=self.device)
+                                    if mats else None)
 
     def add_matrix(self, name: str, W: torch.Tensor, act_rms: torch.Tensor, sign_seed: int = q.DEFAULT_SIGN_SEED):
         spec, dev = self.spec, self.device
@@ -174,6 +177,8 @@ class ModelCodec:
             cur.wait_event(st.record_event())
 
     def calibrate_all(self):
+        if self.use_batch and self.batch is not None:
+            return self.batch.calibrate(self.batch_workspace, self.status)
         self._phase(lambda s, ws, st: q.calibrate(s.W, s.params, s.chan_scale, s.signs, s.sigma, ws, self.status, st))
 
     def encode_all(self):
@@ -189,6 +194,8 @@ class ModelCodec:
                                                s.params, s.w_hat, st))
 
     def distortion_all(self):
+        if self.use_batch and self.batch is not None:
+            return self.batch.distortion()
         self._phase(lambda s, ws, st: q.distortion(s.W, s.w_hat, s.act_rms, s.params, s.dist, st))
 
     def step(self):
@@ -219,9 +226,21 @@ class ModelCodec:
         # class of row lengths (rows of up to 11264 elements, longer rows)
         n = len(self.slots)
         if self.use_batch and self.batch is not None:
-            enc = len({s.d_in > 11264 for s in self.slots})
-            return 3 * n + enc + 1
+            # one encoder block size per class of row lengths; calibration = one pass and one finish launch
+            # per class; distortion = a zeroing launch and the batch kernel; one decode launch
+            classes = len({self._encoder_class(s.d_in) for s in self.slots})
+            return 2 * classes + classes + 1 + 2
         return 5 * n
+
+    @staticmethod
+    def _encoder_class(d_in: int) -> int:
+        n_seg = (d_in + 511) // 512
+        best, busy = 0, 0
+        for w in (20, 24, 28):
+            b = min(15, w // n_seg) * n_seg
+            if b > busy:
+                best, busy = w, b
+        return best
 
     def totals(self, group=None) -> Dict[str, float]:
         """Error figures over all matrices of all ranks (see combine_distortion)."""
