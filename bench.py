@@ -237,7 +237,10 @@ def run_ours(args):
 
     spec = synth.workload(args.workload, args.K or None, args.block or None)
     layers = list(range(min(args.layers, spec.n_layers))) if args.layers else None
+    t0 = time.perf_counter()
     cb_host, train_mse = q.train_codebook(spec.K)
+    train_host_s = time.perf_counter() - t0
+    gpu_train = q.train_codebook_gpu(spec.K) if rank == 0 else None  # same rules on the device; timed, not used below
     mc = ModelCodec.from_synthetic(spec, dev, cb_host, rank=rank, layers=layers)
     n_w = mc.n_weights
     enc_bytes, dec_bytes = mc.algorithmic_bytes()
@@ -278,9 +281,11 @@ def run_ours(args):
     totals = mc.totals()
 
     # ---- end-to-end: inputs in pinned host memory, packed stream read back -----------------------
-    e2e = None
+    e2e = e2e_full = None
     if not args.no_e2e:
         e2e = run_e2e(mc, args, world, dist if world > 1 else None)
+        if world == 1:
+            e2e_full = run_e2e(mc, args, world, None, with_reconstruction=True)
 
     if rank != 0:
         if world > 1:
@@ -288,7 +293,10 @@ def run_ours(args):
         return
 
     peak, peak_kind = measured_peaks()
-    n_launch = len(mc.slots)
+    enc_launches = len({mc._encoder_class(s.d_in) for s in mc.slots}) if mc.use_batch else len(mc.slots)
+    dec_launches = 1 if mc.use_batch else len(mc.slots)
+    fp32_peak = q.measure_fp32_peak()
+    pipe = load_pipe_note()
     enc_gbs = enc_bytes / (enc_ms * 1e-3) / 1e9
     dec_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
     out = {
@@ -303,6 +311,12 @@ def run_ours(args):
                    "step": "calibrate + encode + decode + distortion, phase by phase over all matrices",
                    "table": {"grid": int(mc.codebook.table_info()[0]), "bytes": int(mc.codebook.table_info()[5])},
                    "codebook_train_mse": train_mse},
+        "codebook_training": {"K": spec.K, "samples": 1 << 20, "host_s": train_host_s,
+                              "device_s": gpu_train["seconds"], "device_updates": gpu_train["iters"],
+                              "device_vs_host_max_abs_diff": float(np.abs(gpu_train["codebook"] - cb_host).max()),
+                              "paper": "about 5 s per bitrate level, hardware not stated (Limitations section)"},
+        "fp32_issue_peak": {"lane_inst_per_s": fp32_peak, "tflops_as_fma": 2 * fp32_peak / 1e12,
+                            "how": "qamw_measure_fp32_peak: FMA kernel, eight independent chains per thread"},
         "encode_gweights_s": world * n_w / (enc_ms * 1e-3) / 1e9,
         "decode_gb_s": world * dec_gbs,
         "phases_ms": {"calibrate": cal_ms, "encode": enc_ms, "decode": dec_ms, "distortion": dis_ms},
@@ -310,23 +324,35 @@ def run_ours(args):
         "gpu_launches": mc.kernel_launches_per_step() * args.steps,
         "roofline": {"kernel": "encode2_kernel", "bound": "hbm", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
                      "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": enc_gbs / 8000.0,
-                     "algorithmic_bytes_per_launch": enc_bytes / n_launch, "avg_launch_ms": enc_ms / n_launch,
-                     "traffic": None},
+                     "algorithmic_bytes_per_launch": enc_bytes / enc_launches, "avg_launch_ms": enc_ms / enc_launches,
+                     "launches_per_step": enc_launches, "traffic": None},
         "roofline_decode": {"kernel": "decode2_kernel", "bound": "hbm", "achieved": dec_gbs, "peak": peak,
                             "unit": "GB/s", "frac": dec_gbs / peak, "peak_kind": f"of {peak_kind}",
                             "frac_of_nominal_8TBs": dec_gbs / 8000.0,
-                            "algorithmic_bytes_per_launch": dec_bytes / n_launch, "avg_launch_ms": dec_ms / n_launch,
-                            "traffic": None},
+                            "algorithmic_bytes_per_launch": dec_bytes / dec_launches, "avg_launch_ms": dec_ms / dec_launches,
+                            "launches_per_step": dec_launches, "traffic": None},
         "quality": totals, "status_word": status_word, "wall_s_timed_region": t_wall,
     }
     if e2e is not None:
         out["e2e"] = e2e
+    if e2e_full is not None:
+        out["e2e_with_reconstruction"] = e2e_full
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(spec, golden_or_trained_codebook(spec.K), args)
     traffic = load_traffic_note()
     if traffic:  # measured bytes per weight x weights of the average launch
-        out["roofline"]["traffic"] = traffic["encode"] * n_w / n_launch
-        out["roofline_decode"]["traffic"] = traffic["decode"] * n_w / n_launch
+        out["roofline"]["traffic"] = traffic["encode"] * n_w / enc_launches
+        out["roofline_decode"]["traffic"] = traffic["decode"] * n_w / dec_launches
+    if pipe and clocks and clocks.get("sm_mhz"):
+        # The encoder is bound by the shared-memory / load-store data pipe, not by HBM: one wavefront per
+        # clock per SM is that pipe's peak, and ncu counted how many wavefronts a 2-D point costs.
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        wf_s = pipe["encode_lsu_wavefronts_per_point"] * (n_w / 2) / (enc_ms * 1e-3)
+        pk = sms * clocks["sm_mhz"] * 1e6
+        out["roofline_encode_pipe"] = {"kernel": "encode2_kernel", "bound": "lsu (shared-memory data pipe)",
+                                       "achieved": wf_s / 1e9, "peak": pk / 1e9, "unit": "Gwavefronts/s",
+                                       "frac": wf_s / pk, "wavefronts_per_point": pipe["encode_lsu_wavefronts_per_point"],
+                                       "source": "profiles/encode_pipe.txt (ncu l1tex__data_pipe_lsu_wavefronts)"}
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -344,7 +370,7 @@ def load_traffic_note():
                 if line.strip() and not line.startswith("#"):
                     k, v = line.split()[:2]
                     note[k] = v
-        src = os.path.join(ROOT, "paper_2605_26339_b200", "csrc", "qamw_kernels.cu")
+        src = os.path.join(ROOT, "paper_2605_26339_b200", "csrc", "qamw_rows.cu")
         with open(src, "rb") as f:
             if hashlib.sha256(f.read()).hexdigest() != note.get("kernel_source_sha256"):
                 return None
@@ -354,7 +380,26 @@ def load_traffic_note():
         return None
 
 
-def run_e2e(mc, args, world, dist):
+def load_pipe_note():
+    """Load/store-pipe wavefronts per 2-D point of the encoder, counted once with ncu
+    (profiles/encode_pipe.txt, same format and staleness rule as the traffic note)."""
+    import hashlib
+    try:
+        note = {}
+        with open(os.path.join(ROOT, "profiles", "encode_pipe.txt")) as f:
+            for line in f:
+                if line.strip() and not line.startswith("#"):
+                    k, v = line.split()[:2]
+                    note[k] = v
+        with open(os.path.join(ROOT, "paper_2605_26339_b200", "csrc", "qamw_rows.cu"), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != note.get("kernel_source_sha256"):
+                return None
+        return {"encode_lsu_wavefronts_per_point": float(note["encode_lsu_wavefronts_per_point"])}
+    except Exception:
+        return None
+
+
+def run_e2e(mc, args, world, dist, with_reconstruction=False):
     """The same step driven from pinned host memory: every matrix is copied host -> device, then
     calibrated, encoded, decoded and scored; the packed stream, row norms and distortion sums are
     copied back.  Copies run on their own streams and overlap the kernels."""
@@ -377,10 +422,16 @@ def run_e2e(mc, args, world, dist):
     for s in slots[:per_layer]:
         out_bufs[(s.d_out, s.d_in)] = (torch.empty(s.packed.shape, dtype=torch.uint8, pin_memory=True),
                                        torch.empty(s.row_norm.shape, dtype=torch.float32, pin_memory=True))
+    what_bufs = {}
+    if with_reconstruction:
+        for s in slots[:per_layer]:
+            what_bufs[(s.d_out, s.d_in)] = torch.empty(s.w_hat.shape, dtype=torch.bfloat16, pin_memory=True)
     dist_host = torch.empty((len(slots), 4), dtype=torch.float64, pin_memory=True)
     h2d, comp, d2h = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
     h2d_bytes = sum(s.W.numel() * s.W.element_size() for s in slots)
     d2h_bytes = sum(s.packed.numel() + 4 * s.row_norm.numel() + 32 for s in slots)
+    if with_reconstruction:
+        d2h_bytes += sum(2 * s.w_hat.numel() for s in slots)
 
     def one_step():
         for i, s in enumerate(slots):
@@ -402,6 +453,8 @@ def run_e2e(mc, args, world, dist):
                 pk.copy_(s.packed, non_blocking=True)
                 nm.copy_(s.row_norm, non_blocking=True)
                 dist_host[i].copy_(s.dist, non_blocking=True)
+                if with_reconstruction:
+                    what_bufs[(s.d_out, s.d_in)].copy_(s.w_hat, non_blocking=True)
 
     def barrier():
         torch.cuda.synchronize()
@@ -410,7 +463,7 @@ def run_e2e(mc, args, world, dist):
 
     one_step()
     barrier()
-    steps = max(1, min(args.steps, 3))
+    steps = max(1, min(args.steps, 2 if with_reconstruction else 3))
     t0 = time.perf_counter()
     for _ in range(steps):
         one_step()
@@ -422,8 +475,11 @@ def run_e2e(mc, args, world, dist):
     sec = float(t.cpu()[0])
     return {"value": world * mc.n_weights / sec / 1e9, "unit": "Gweights/s", "h2d_bytes_per_step": h2d_bytes,
             "d2h_bytes_per_step": d2h_bytes, "ms_per_step": sec * 1e3, "steps": steps, "host_layers": host_layers,
-            "note": "weights from pinned host memory; packed stream, row norms and distortion sums read back; "
-                    "the bf16 reconstruction stays on the device, where the paper's pipeline consumes it"}
+            "note": ("weights from pinned host memory; packed stream, row norms, distortion sums and the decoded bf16 "
+                     "matrices read back" if with_reconstruction else
+                     "encode side end to end: weights from pinned host memory; packed stream, row norms and distortion "
+                     "sums read back; the bf16 reconstruction stays on the device, where the paper's pipeline consumes "
+                     "it (e2e_with_reconstruction also copies it back)")}
 
 
 def cpu_baseline(spec, cb_host, args):

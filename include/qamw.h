@@ -279,6 +279,27 @@ int qamw_round_f16(float* values, size_t n, void* stream);
 int qamw_renorm_row_norms(const uint8_t* packed, const float* row_norm, const float* sigma, const qamw_codebook* cb,
                           const qamw_params* p, float* row_norm_out, void* stream);
 
+/* Fused decode -> matrix-vector product (the paper's Section 1 and Limitations name the fused
+ * dequantise-matmul kernel as future work; its own pipeline writes W_hat in BF16 first):
+ *     y[i, v] = sum_j W_hat[i, j] x[v, j],   W_hat the decoder's output of Section 3.2 / B.2 before
+ * its rounding to bf16.  Because the rotation is orthonormal and symmetric (Lemma 1),
+ * w_hat_i . x = r_i sum_k c_idx_k . (sigma_k xt_k) with xt = F S (x / s): the activation is rotated once
+ * per call and no row is ever rotated back or written out.
+ * x: device, n_vec vectors of d_in floats (n_vec in {1, 2, 4}); y_out: device, [d_out, n_vec] floats;
+ * workspace: device, qamw_gemv_workspace_bytes(p, n_vec) bytes, 8-byte aligned.  d_in must be a
+ * multiple of 32 (QAMW_ERR_SHAPE) and the rotated activations must fit in shared memory next to the
+ * codebook (QAMW_ERR_NOMEM).  f32 accumulation; asynchronous on `stream`. */
+size_t qamw_gemv_workspace_bytes(const qamw_params* p, int n_vec);
+int qamw_decode_gemv(const uint8_t* packed, const float* row_norm, const float* chan_scale, const int8_t* signs,
+                     const float* sigma, const qamw_codebook* cb, const qamw_params* p, const float* x, int n_vec,
+                     float* y_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Measures the device's plain FP32 issue rate with a fused-multiply-add kernel (eight independent
+ * chains per thread): lane instructions per second, i.e. half the FMA FLOP/s.  This is the roofline an
+ * exhaustive nearest-codeword search (QAMW_FLAG_BRUTE_FORCE) is bound by; the paper gives no such
+ * figure.  scratch_dev: device, one float.  Synchronous (times its own launch with events). */
+int qamw_measure_fp32_peak(float* scratch_dev, double* lane_inst_per_s_out);
+
 /* Corollary 3 / Corollary 4 sums in double:
  *   out4[0] = sum (W - W_hat)^2        out4[1] = sum W^2
  *   out4[2] = sum r_j^2 (W - W_hat)^2  out4[3] = sum r_j^2 W^2     (r_j = act_rms, 1 if NULL)

@@ -35,7 +35,7 @@ EXPORTED = [
     "qamw_distortion", "qamw_last_cuda_error",
     "qamw_batch_create", "qamw_batch_destroy", "qamw_batch_workspace_bytes", "qamw_calibrate_batch",
     "qamw_encode_batch", "qamw_decode_batch", "qamw_distortion_batch",
-    "qamw_quantize", "qamw_train_codebook_gpu", "qamw_round_f16", "qamw_renorm_row_norms", "qamw_polar_train", "qamw_polar_codebook", "qamw_codebook_create_polar",
+    "qamw_quantize", "qamw_gemv_workspace_bytes", "qamw_decode_gemv", "qamw_measure_fp32_peak", "qamw_train_codebook_gpu", "qamw_round_f16", "qamw_renorm_row_norms", "qamw_polar_train", "qamw_polar_codebook", "qamw_codebook_create_polar",
 ]
 
 
@@ -96,6 +96,10 @@ def lib() -> C.CDLL:
         L.qamw_last_cuda_error.restype = C.c_char_p
         L.qamw_train_codebook_gpu.argtypes = [i32, u64, u64, vp, i32, C.c_double, vp, vp, vp, vp, vp]
         L.qamw_quantize.argtypes = [vp, C.POINTER(Params), vp, C.c_float, u64, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.qamw_gemv_workspace_bytes.argtypes = [C.POINTER(Params), i32]
+        L.qamw_gemv_workspace_bytes.restype = sz
+        L.qamw_decode_gemv.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Params), vp, i32, vp, vp, sz, vp]
+        L.qamw_measure_fp32_peak.argtypes = [vp, vp]
         L.qamw_round_f16.argtypes = [vp, sz, vp]
         L.qamw_renorm_row_norms.argtypes = [vp, vp, vp, vp, C.POINTER(Params), vp, vp]
         L.qamw_polar_train.argtypes = [i32, vp, vp]
@@ -357,6 +361,25 @@ def decode(packed: torch.Tensor, row_norm: torch.Tensor, chan_scale, signs, sigm
            w_hat_out: torch.Tensor, stream=None):
     _check("qamw_decode", lib().qamw_decode(_dp(packed), _dp(row_norm), _dp(chan_scale), _dp(signs), _dp(sigma),
                                            cb.handle, C.byref(p), _dp(w_hat_out), _stream(stream)))
+
+
+def decode_gemv(packed: torch.Tensor, row_norm: torch.Tensor, chan_scale, signs, sigma, cb: Codebook, p: Params,
+                x: torch.Tensor, y_out: torch.Tensor, workspace: Optional[torch.Tensor] = None, stream=None):
+    """y = W_hat x straight from the packed stream (x: float32 [n_vec, d_in], y_out: float32 [d_out, n_vec])."""
+    n_vec = x.shape[0]
+    if workspace is None:
+        workspace = torch.empty(int(lib().qamw_gemv_workspace_bytes(C.byref(p), n_vec)), dtype=torch.uint8, device=x.device)
+    _check("qamw_decode_gemv", lib().qamw_decode_gemv(
+        _dp(packed), _dp(row_norm), _dp(chan_scale), _dp(signs), _dp(sigma), cb.handle, C.byref(p), _dp(x), n_vec,
+        _dp(y_out), _dp(workspace), workspace.numel(), _stream(stream)))
+
+
+def measure_fp32_peak() -> float:
+    """Plain FP32 lane instructions per second of the current device (FMA micro-benchmark)."""
+    scratch = torch.zeros(1, dtype=torch.float32, device="cuda")
+    out = C.c_double()
+    _check("qamw_measure_fp32_peak", lib().qamw_measure_fp32_peak(_dp(scratch), C.addressof(out)))
+    return out.value
 
 
 def round_f16(values: torch.Tensor, stream=None):

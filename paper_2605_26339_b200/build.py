@@ -8,7 +8,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 _INC = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.path.join(_PKG, "libqamw.so")
-SOURCES = ["qamw_kernels.cu", "qamw_rows.cu", "qamw_lloyd.cu", "qamw_variants.cu", "qamw_host.cpp", "qamw_table.cpp"]
+SOURCES = ["qamw_kernels.cu", "qamw_rows.cu", "qamw_lloyd.cu", "qamw_variants.cu", "qamw_gemv.cu", "qamw_host.cpp", "qamw_table.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-Wall,-Wextra", "-shared"]
 

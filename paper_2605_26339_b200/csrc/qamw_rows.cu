@@ -760,22 +760,40 @@ __global__ void __launch_bounds__(MAXT, 1) encode2_kernel(const Encode2Args a) {
 }
 
 // sigma_k of every matrix from the slots of partial sums (zeroed before the calibration pass, so a
-// slot nobody wrote counts as empty): thread = one pair position, slots added in ascending order.
-__global__ void calibrate_finish2_kernel(const MatDesc* descs, const unsigned char* calib_base) {
+// slot nobody wrote counts as empty).  A block owns 32 pair positions of one matrix; its eight
+// warps each add a contiguous slice of the slots in ascending order, and the eight slice sums are
+// then added in ascending order: the result does not depend on timing.
+constexpr int kFinishSlices = 8;
+__global__ void __launch_bounds__(32 * kFinishSlices) calibrate_finish2_kernel(const MatDesc* descs,
+                                                                             const unsigned char* calib_base) {
+    __shared__ double part_sum[kFinishSlices][32], part_used[kFinishSlices];
     const MatDesc& d = descs[blockIdx.y];
     const int n_pairs = d.d_in >> 1, pair_stride = (n_pairs + 3) & ~3;
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= n_pairs) return;
+    if (int(blockIdx.x) * 32 >= n_pairs) return;
+    const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
+    const int k = blockIdx.x * 32 + lane;
     const double* ws = reinterpret_cast<const double*>(calib_base + d.calib_offset);
-    double s = 0.0, u = 0.0;
-    for (int slot = 0; slot < d.calib_slots; ++slot) {
-        s += ws[size_t(slot) * pair_stride + k];
-        u += ws[size_t(d.calib_slots) * pair_stride + slot];
+    const int per = (d.calib_slots + kFinishSlices - 1) / kFinishSlices;
+    const int s0 = min(d.calib_slots, slice * per), s1 = min(d.calib_slots, s0 + per);
+    double sum = 0.0, used = 0.0;
+    for (int slot = s0; slot < s1; ++slot) {
+        if (k < n_pairs) sum += ws[size_t(slot) * pair_stride + k];
+        if (lane == 0) used += ws[size_t(d.calib_slots) * pair_stride + slot];
     }
-    const double inv_sqrt_d = 1.0 / sqrt(double(d.d_in));
-    double sg = u > 0.0 ? (s / u) / sqrt(1.5707963267948966) : inv_sqrt_d;  // Rayleigh mean = sigma sqrt(pi / 2)
-    sg = fmax(sg, 1e-4 * inv_sqrt_d);
-    const_cast<float*>(d.sigma)[k] = float(sg);
+    part_sum[slice][lane] = sum;
+    if (lane == 0) part_used[slice] = used;
+    __syncthreads();
+    if (slice == 0 && k < n_pairs) {
+        double s = 0.0, u = 0.0;
+        for (int i = 0; i < kFinishSlices; ++i) {
+            s += part_sum[i][lane];
+            u += part_used[i];
+        }
+        const double inv_sqrt_d = 1.0 / sqrt(double(d.d_in));
+        double sg = u > 0.0 ? (s / u) / sqrt(1.5707963267948966) : inv_sqrt_d;  // Rayleigh mean = sigma sqrt(pi / 2)
+        sg = fmax(sg, 1e-4 * inv_sqrt_d);
+        const_cast<float*>(d.sigma)[k] = float(sg);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1241,8 +1259,8 @@ extern "C" int qamw_calibrate_batch(const qamw_batch* b, void* workspace, size_t
             if (rc == QAMW_OK) {
                 int max_pairs = 0;
                 for (const MatDesc& d : set.descs) max_pairs = std::max(max_pairs, d.d_in / 2);
-                calibrate_finish2_kernel<<<dim3(unsigned((max_pairs + 255) / 256), unsigned(set.descs.size())), 256, 0, st>>>(
-                    set.d_descs, ws);
+                calibrate_finish2_kernel<<<dim3(unsigned((max_pairs + 31) / 32), unsigned(set.descs.size())),
+                                           32 * kFinishSlices, 0, st>>>(set.d_descs, ws);
                 rc = launch_check("calibrate_finish2_kernel");
             }
         }

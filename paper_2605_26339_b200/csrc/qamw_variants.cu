@@ -77,3 +77,46 @@ extern "C" int qamw_renorm_row_norms(const uint8_t* packed, const float* row_nor
         p->d_in / 2, row_norm_out);
     return launched("renorm_kernel");
 }
+
+// ---------------------------------------------------------------------------------------------
+// FP32 issue-rate probe: the plain-ALU roofline that an exhaustive search would be measured against
+// ---------------------------------------------------------------------------------------------
+namespace {
+__global__ void __launch_bounds__(256) fma_probe_kernel(float* out, int iters, float a, float b) {
+    float x[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = float(threadIdx.x + i);
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int u = 0; u < 16; ++u)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = fmaf(x[i], a, b);  // eight independent chains
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s += x[i];
+    if (s == 12345.678f) out[0] = s;  // never true: keeps the chains alive
+}
+}  // namespace
+
+extern "C" int qamw_measure_fp32_peak(float* scratch_dev, double* lane_inst_per_s_out) {
+    if (!scratch_dev || !lane_inst_per_s_out) return QAMW_ERR_ARG;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return QAMW_ERR_CUDA;
+    const int blocks = 8 * sm_count(), iters = 4096;
+    fma_probe_kernel<<<blocks, 256>>>(scratch_dev, 64, 1.0000001f, 1e-9f);  // warm-up
+    cudaEventRecord(e0);
+    fma_probe_kernel<<<blocks, 256>>>(scratch_dev, iters, 1.0000001f, 1e-9f);
+    cudaEventRecord(e1);
+    cudaError_t e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (e != cudaSuccess || !(ms > 0.f)) {
+        set_cuda_error("qamw_measure_fp32_peak", int(e));
+        return QAMW_ERR_CUDA;
+    }
+    *lane_inst_per_s_out = double(blocks) * 256.0 * double(iters) * 128.0 / (double(ms) * 1e-3);
+    return QAMW_OK;
+}

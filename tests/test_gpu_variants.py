@@ -125,3 +125,43 @@ def test_alpha_grid_picks_the_lowest_output_error(orc):
     what = orc.decode(enc["packed"], enc["row_norm"], 128, cb.host, s, signs, sigma, 1024)
     d = orc.distortion(Wb, what, act)
     assert abs(np.sqrt(d[2] / d[3]) - scores[0.5][1]) < 2e-3 * scores[0.5][1]
+
+
+@pytest.mark.parametrize("d_out,d_in,block,K,n_vec", [(300, 2048, 128, 2048, 1), (129, 5120, 128, 256, 4),
+                                                      (64, 13824, 256, 2048, 2), (40, 1024, 32, 128, 1),
+                                                      (33, 512, 1024 // 2, 4096, 1)])
+def test_fused_decode_gemv(orc, d_out, d_in, block, K, n_vec):
+    """y = W_hat x from the packed stream against the oracle's decoder (f64, before the bf16 rounding)
+    followed by a plain matrix product.  The kernel accumulates in f32: the error of a row stays below
+    1e-5 |w_hat_i| |x| (d_in terms, each product and sum rounded to 2^-24 relative)."""
+    W, act = _problem(50 + n_vec, d_out, d_in)
+    e = _encode(W, act, 0.3, block, K)
+    g = torch.Generator().manual_seed(d_in)
+    x = torch.randn((n_vec, d_in), generator=g)
+    y = torch.full((d_out, n_vec), float("nan"), dtype=torch.float32, device=DEV)
+    q.decode_gemv(e["packed"], e["norm"], e["s"], e["signs"], e["sigma"], e["cb"], e["p"], x.to(DEV), y)
+    _, w64 = orc.decode(e["packed"].cpu().numpy(), e["norm"].cpu().numpy(), block, e["cbh"], e["s"].cpu().numpy(),
+                        e["signs"].cpu().numpy(), e["sigma"].cpu().numpy(), d_in, want_f64=True)
+    ref = w64 @ x.numpy().astype(np.float64).T
+    bound = 1e-5 * np.sqrt((w64 ** 2).sum(1))[:, None] * np.sqrt((x.numpy().astype(np.float64) ** 2).sum(1))[None, :]
+    assert np.all(np.abs(y.cpu().numpy() - ref) <= bound + 1e-30)
+    # and against the two-step pipeline of the paper (decode to bf16, then multiply): bf16 rounding only
+    what = torch.empty((d_out, d_in), dtype=torch.bfloat16, device=DEV)
+    q.decode(e["packed"], e["norm"], e["s"], e["signs"], e["sigma"], e["cb"], e["p"], what)
+    two_step = what.double() @ x.to(DEV).double().T
+    assert torch.allclose(y.double(), two_step, rtol=0, atol=float(2.0 ** -7 * np.abs(ref).max() + 1e-30))
+
+
+def test_fused_gemv_argument_errors():
+    lv = load_golden_codebook(64)
+    cb = q.Codebook(lv)
+    dummy = torch.zeros(4096, dtype=torch.uint8, device=DEV)
+    f = torch.zeros(4096, dtype=torch.float32, device=DEV)
+    p = q.make_params(None, 4, 48, 16, 64)  # d_in not a multiple of 32
+    with pytest.raises(q.QamwError) as e:
+        q.decode_gemv(dummy, f, None, dummy, f, cb, p, f[:48].reshape(1, 48), f[:4].reshape(4, 1), dummy)
+    assert e.value.code == q.ERR_SHAPE
+    p = q.make_params(None, 4, 64, 16, 64)
+    with pytest.raises(q.QamwError) as e:
+        q.decode_gemv(dummy, f, None, dummy, f, cb, p, f[:192].reshape(3, 64), f[:12].reshape(4, 3), dummy)  # 3 vectors
+    assert e.value.code == q.ERR_ARG

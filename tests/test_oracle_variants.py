@@ -37,3 +37,23 @@ def test_renormalised_decode_restores_the_row_norm(orc):
     # same direction either way
     cos = (plain * renorm).sum(1) / np.sqrt((plain ** 2).sum(1) * (renorm ** 2).sum(1))
     assert np.allclose(cos, 1.0, atol=1e-12)
+
+
+def test_fused_product_identity(orc):
+    """The identity behind the fused decode -> matrix-vector product (Lemma 1: the block Hadamard
+    matrix is symmetric and orthonormal): w_hat_i . x = r_i sum_k c_idx_k . (sigma_k xt_k) with
+    xt = R_fwd (x / s), checked with the oracle's decoder and forward rotation."""
+    rng = np.random.default_rng(8)
+    d_out, d_in, b, K = 6, 256, 64, 32
+    W = rng.standard_normal((d_out, d_in)).astype(np.float32)
+    act = np.exp(rng.standard_normal(d_in)).astype(np.float32)
+    s = orc.channel_scales(act, 0.3)
+    signs = orc.make_signs(3, d_in)
+    sigma, _ = orc.calibrate(W, b, s, signs)
+    cb = orc.train_codebook(K, 1 << 12, 1, 20, 1e-5)[0]
+    enc = orc.encode(W, b, cb, s, signs, sigma, diagnostics=True)
+    _, what = orc.decode(enc["packed"], enc["row_norm"], b, cb, s, signs, sigma, d_in, want_f64=True)
+    x = rng.standard_normal(d_in)
+    xt = orc.rotate_fwd(x / s.astype(np.float64), signs, b).reshape(-1, 2) * sigma.astype(np.float64)[:, None]
+    fused = enc["row_norm"].astype(np.float64) * (cb[enc["idx"]].astype(np.float64) * xt[None]).sum((1, 2))
+    assert np.allclose(fused, what @ x, rtol=1e-12, atol=1e-12)
