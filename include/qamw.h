@@ -66,7 +66,7 @@ extern "C" {
 #define QAMW_DEFAULT_SIGN_SEED 0x51A5C0DEC0FFEE01ULL
 #define QAMW_MAX_BLOCK 1024 /* cap of Section 3.3 */
 #define QAMW_MAX_K 4096
-#define QAMW_CALIB_MAX_ROWS 1024 /* "up to 1024 unit-normalized rows" (Section 3.4) */
+#define QAMW_CALIB_MAX_ROWS 1024 /* row cap of the sigma calibration (Section 3.4) */
 #define QAMW_STATIC_SCRATCH_BYTES (16u << 20) /* built-in scratch of qamw_calibrate_static */
 
 typedef struct {
@@ -85,7 +85,7 @@ typedef struct qamw_codebook qamw_codebook; /* opaque: device copy of C plus its
  * Host-side helpers (host pointers only, no CUDA calls).
  * -------------------------------------------------------------------------------------------- */
 
-/* Section 3.6: "trained by Lloyd iterations on the unit circular Gaussian".  Sample-based Lloyd
+/* Section 3.6: the codebook is the Lloyd-Max quantiser of the unit circular Gaussian.  Sample-based Lloyd
  * on n_samples Box-Muller samples of counter stream `seed` (u = ((mix64(mix64(seed ^
  * 0xD1B54A32D192ED03) + golden*(n+1)) >> 11) + 0.5) * 2^-53, sample i from counters 2i, 2i+1);
  * initial codewords sqrt(2) * sample_i; each iteration assigns every sample to its nearest
@@ -119,7 +119,7 @@ int qamw_train_codebook_gpu(int K, uint64_t n_samples, uint64_t seed, const doub
  * alpha == 0 gives all ones.  act_rms, s_out: host, d_in floats. */
 int qamw_channel_scales(const float* act_rms, int d_in, float alpha, float* s_out);
 
-/* Sign mask of Appendix A.1 ("deterministic sequence generated from a fixed 64-bit seed"):
+/* Sign mask of Appendix A.1 (a fixed sequence derived from one 64-bit seed):
  * sign_j = -1 if the top bit of mix64(seed + 0x9E3779B97F4A7C15*(j+1)) is set, else +1, with
  * mix64 the SplitMix64 finaliser.  signs_out: host, d_in bytes of +1 / -1. */
 int qamw_make_signs(uint64_t seed, int d_in, int8_t* signs_out);
@@ -142,8 +142,8 @@ int qamw_status_to_error(int32_t status_word);
  * -------------------------------------------------------------------------------------------- */
 
 /* Uploads the K x 2 f32 codebook (host pointer) to the current device and builds the exact
- * spatial search table used by qamw_encode (Section 3.6: "nearest codebook entry by Euclidean
- * distance"): the plane is cut into grid x grid cells, narrow where a Gaussian source puts its
+ * spatial search table used by qamw_encode (Section 3.6: the Euclidean-nearest
+ * codeword): the plane is cut into grid x grid cells, narrow where a Gaussian source puts its
  * codewords and widening outwards; every cell lists all codewords whose nearest-neighbour region
  * can meet the cell, so a scan of the list returns what a scan of the whole codebook returns.
  * The outermost cells reach to |z| < 16384; points beyond are scanned exhaustively.  grid = 0
@@ -267,8 +267,8 @@ int qamw_decode(const uint8_t* packed, const float* row_norm, const float* chan_
                 void* w_hat_bf16_out, void* stream);
 
 /* Variants around the path.
- * qamw_round_f16 (Section 3.2: the bitrate charges 16 bits per row norm and per channel scale; "a
- * fully serialized f16 row norm" adds a radial quantisation term): rounds n f32 values on the device,
+ * qamw_round_f16 (Section 3.2: the bitrate charges 16 bits per row norm and per channel scale; storing
+ * the norm as binary16 adds a radial quantisation term): rounds n f32 values on the device,
  * in place, to IEEE binary16 (nearest even) and back.  Round channel scales and sigma before
  * qamw_encode, row norms after it, and decode sees exactly what a 16-bit serialisation would hold.
  * qamw_renorm_row_norms (Section A.3, the optional final direction renormalisation): writes

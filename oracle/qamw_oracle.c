@@ -15,8 +15,8 @@
  *     order (see orc_front_row), so that a second implementation can reproduce
  *     the exact bits of the 2-D points that the nearest-codeword decision sees.
  *   - Nearest-codeword search is exhaustive over all K codewords, in double,
- *     lowest index wins exact ties (Section 3.6, "nearest codebook entry by
- *     Euclidean distance").
+ *     lowest index wins exact ties (Section 3.6: the Euclidean-nearest
+ *     codeword).
  *
  * Parity pins live in tests/test_oracle_*.py.  Unpinned by the paper (pinned only
  * by this repository's own written specification): the sign-mask generator, the
@@ -45,7 +45,7 @@ int orc_num_threads(void) {
 
 /* ------------------------------------------------------------------------- */
 /* Counter-based generators (repository specification; the paper only says     */
-/* "a deterministic sequence generated from a fixed 64-bit seed", Section A.1, */
+/* A fixed sequence derived from one 64-bit seed (Section A.1,                */
 /* Definition "Sign mask").                                                   */
 /* ------------------------------------------------------------------------- */
 
@@ -275,7 +275,7 @@ void orc_fwht_f64(double *x, int b) {
  *   (iii) h   = butterfly_f32(x) per block of b   (orc_fwht_f32)
  *   (iv)  c_b = f32( 1 / sqrt((double)b) );  g = f32( c_b / r )  (one f32 division)
  *         y_j = f32(h_j * g)
- *         r == 0  ->  y = 0   (Section 3.1 step 1: "encoded as a zero row")
+ *         r == 0  ->  y = 0   (Section 3.1 step 1: a zero row encodes as zeros)
  * Returns ORC_ERR_NONFINITE when r is not finite (y is then unspecified).
  */
 int orc_front_row(const void *W_row, int w_dtype, int d_in, int b, const float *chan_scale,
@@ -711,7 +711,7 @@ double orc_rayleigh_distortion(const double *levels, int n) {
 
 /* N-level Lloyd-Max quantiser of the unit Rayleigh density under squared error:
  * start from the quantiles r_j = sqrt(-2 ln(1 - (j + 1/2)/N)), then alternate
- * "cell boundaries = midpoints of the levels" and "level = centroid of its cell"
+ * cell boundaries at the midpoints of the levels, every level at the centroid of its cell
  * (numerically integrated on [0, 8]) until no level moves by more than 1e-13 or
  * max_iters rounds.  levels_out: f32 (the practical codebook); returns the
  * numerically integrated distortion C_LM of those f32 levels. */
@@ -853,7 +853,7 @@ int orc_encode_polar(const void *W, int w_dtype, int d_out, int d_in, int64_t w_
 /* Variants around the path.                                                   */
 /* ------------------------------------------------------------------------- */
 
-/* Section 3.2: "a fully serialized f16 row norm" -- metadata rounded to IEEE
+/* Section 3.2: the row norm serialised as binary16 -- metadata rounded to IEEE
  * binary16 (nearest even; overflow to infinity, gradual underflow) and widened
  * back to f32, in place. */
 void orc_round_f16(float *v, int64_t n) {
