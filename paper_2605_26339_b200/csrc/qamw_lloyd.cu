@@ -238,6 +238,8 @@ extern "C" int qamw_train_codebook_gpu(int K, uint64_t n_samples, uint64_t seed,
     for (int c = 0; c < 2 * K; ++c) cb[size_t(c)] = root2 * first[size_t(c)];
     ok(cudaMemcpy(d_cb, cb.data(), sizeof(double) * 2 * K, cudaMemcpyHostToDevice));
     std::vector<double> err(size_t(assign_blocks), 0.0);
+    if (sizeof(double2) * size_t(K) > 48 * 1024)  // K = 4096: the codebook needs more than the default dynamic limit
+        ok(cudaFuncSetAttribute(assign_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sizeof(double2) * size_t(K))));
     auto assign_pass = [&](bool keep) -> double {
         assign_kernel<<<assign_blocks, kAssignThreads, sizeof(double2) * K>>>(samples, n, d_cb, K, keep ? d_assign : nullptr,
                                                                              d_err);

@@ -19,7 +19,7 @@ if torch.cuda.is_available():
 DEV = "cuda:0"
 
 
-@pytest.mark.parametrize("K,n,iters", [(1, 4096, 3), (2, 5000, 20), (64, 1 << 14, 25), (256, 1 << 16, 12)])
+@pytest.mark.parametrize("K,n,iters", [(1, 4096, 3), (2, 5000, 20), (64, 1 << 14, 25), (256, 1 << 16, 12), (4096, 1 << 15, 4)])
 def test_training_on_the_oracles_samples_reproduces_the_oracle(orc, K, n, iters):
     samples = orc.gauss_pairs(9, n)
     ref_cb, ref_mse, ref_iters, ref_trace = orc.train_codebook(K, n, 9, iters, 1e-7, want_trace=True)

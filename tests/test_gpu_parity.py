@@ -218,7 +218,7 @@ def test_cfg0_full(orc):
     W = synth.make_weight(spec, spec.matrices[0], synth.matrix_seed(spec, 0, 0))
     act = synth.make_act_rms(spec, 1024, 1).numpy()
     rep = Case(orc, W, act, spec.alpha, spec.block, spec.K).check_all()
-    print("cfg0", rep)
+    _report("cfg0 all rows", rep)
 
 
 @pytest.mark.parametrize("kernels", ["fast", "general"])
@@ -350,7 +350,7 @@ def test_full_size_matrices_sampled_rows(orc, name, mid):
     act = synth.make_act_rms(spec, m.d_in, 3, device=DEV).cpu().numpy()
     rows = np.unique(np.concatenate([[0, 1, m.d_out - 1], np.linspace(0, m.d_out - 1, 45).astype(int)]))
     rep = Case(orc, W, act, spec.alpha, spec.block, spec.K, row_sel=rows).check_all()
-    print(name, m.name, rep)
+    _report(f"{name} {m.name} K={spec.K} sampled rows", rep)
 
 
 def test_encode_decode_are_deterministic(orc):
