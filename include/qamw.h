@@ -287,8 +287,12 @@ int qamw_renorm_row_norms(const uint8_t* packed, const float* row_norm, const fl
  * per call and no row is ever rotated back or written out.
  * x: device, n_vec vectors of d_in floats (n_vec in {1, 2, 4}); y_out: device, [d_out, n_vec] floats;
  * workspace: device, qamw_gemv_workspace_bytes(p, n_vec) bytes, 8-byte aligned.  d_in must be a
- * multiple of 32 (QAMW_ERR_SHAPE) and the rotated activations must fit in shared memory next to the
- * codebook (QAMW_ERR_NOMEM).  f32 accumulation; asynchronous on `stream`. */
+ * multiple of 32 (QAMW_ERR_SHAPE).  Packed rows and x that are 16-byte aligned (base and stride) take
+ * the kernel that keeps the rotated activations in registers (one launch, any d_in up to the row-length
+ * limit above); any other layout, or QAMW_FLAG_GENERAL_KERNELS, takes a layout-agnostic pair of kernels
+ * whose rotated activations (n_vec * d_in floats) must fit in shared memory next to the codebook
+ * (QAMW_ERR_NOMEM otherwise).  f32 accumulation in a fixed order: results are reproducible run to run;
+ * asynchronous on `stream`. */
 size_t qamw_gemv_workspace_bytes(const qamw_params* p, int n_vec);
 int qamw_decode_gemv(const uint8_t* packed, const float* row_norm, const float* chan_scale, const int8_t* signs,
                      const float* sigma, const qamw_codebook* cb, const qamw_params* p, const float* x, int n_vec,

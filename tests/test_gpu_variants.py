@@ -129,7 +129,8 @@ def test_alpha_grid_picks_the_lowest_output_error(orc):
 
 @pytest.mark.parametrize("d_out,d_in,block,K,n_vec", [(300, 2048, 128, 2048, 1), (129, 5120, 128, 256, 4),
                                                       (64, 13824, 256, 2048, 2), (40, 1024, 32, 128, 1),
-                                                      (33, 512, 1024 // 2, 4096, 1)])
+                                                      (33, 512, 1024 // 2, 4096, 1), (1000, 2048, 1024, 2048, 4),
+                                                      (7, 64, 2, 64, 2), (50, 11008, 64, 1024, 1)])
 def test_fused_decode_gemv(orc, d_out, d_in, block, K, n_vec):
     """y = W_hat x from the packed stream against the oracle's decoder (f64, before the bf16 rounding)
     followed by a plain matrix product.  The kernel accumulates in f32: the error of a row stays below
@@ -140,11 +141,16 @@ def test_fused_decode_gemv(orc, d_out, d_in, block, K, n_vec):
     x = torch.randn((n_vec, d_in), generator=g)
     y = torch.full((d_out, n_vec), float("nan"), dtype=torch.float32, device=DEV)
     q.decode_gemv(e["packed"], e["norm"], e["s"], e["signs"], e["sigma"], e["cb"], e["p"], x.to(DEV), y)
+    # the layout-agnostic kernel (taken for packed rows that are not 16-byte aligned) gives the same product
+    y_general = torch.full_like(y, float("nan"))
+    pg = q.make_params(None, d_out, d_in, block, K, q.FLAG_GENERAL_KERNELS, e["p"].packed_row_stride)
+    q.decode_gemv(e["packed"], e["norm"], e["s"], e["signs"], e["sigma"], e["cb"], pg, x.to(DEV), y_general)
     _, w64 = orc.decode(e["packed"].cpu().numpy(), e["norm"].cpu().numpy(), block, e["cbh"], e["s"].cpu().numpy(),
                         e["signs"].cpu().numpy(), e["sigma"].cpu().numpy(), d_in, want_f64=True)
     ref = w64 @ x.numpy().astype(np.float64).T
     bound = 1e-5 * np.sqrt((w64 ** 2).sum(1))[:, None] * np.sqrt((x.numpy().astype(np.float64) ** 2).sum(1))[None, :]
     assert np.all(np.abs(y.cpu().numpy() - ref) <= bound + 1e-30)
+    assert np.all(np.abs(y_general.cpu().numpy() - ref) <= bound + 1e-30)
     # and against the two-step pipeline of the paper (decode to bf16, then multiply): bf16 rounding only
     what = torch.empty((d_out, d_in), dtype=torch.bfloat16, device=DEV)
     q.decode(e["packed"], e["norm"], e["s"], e["signs"], e["sigma"], e["cb"], e["p"], what)
