@@ -333,6 +333,7 @@ def run_ours(args):
                             "launches_per_step": dec_launches, "traffic": None},
         "quality": totals, "status_word": status_word, "wall_s_timed_region": t_wall,
     }
+    out["fused_gemv"] = time_fused_gemv(mc, peak)
     if e2e is not None:
         out["e2e"] = e2e
     if e2e_full is not None:
@@ -356,6 +357,51 @@ def run_ours(args):
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_fused_gemv(mc, peak_gbs, calls=50):
+    """y = W_hat x straight from the packed stream (qamw_decode_gemv), one activation vector, every matrix of the
+    first layer in turn so that the packed bytes of a round exceed L2; beside it the paper's pipeline on the same
+    matrices: a bf16 product on the already decoded W_hat (what follows qamw_decode there)."""
+    import torch
+
+    from paper_2605_26339_b200 import binding as q
+    slots = [s for s in mc.slots if s.d_in % 32 == 0][:7]
+    if not slots:
+        return None
+    dev = mc.device
+    xs = [torch.randn((1, s.d_in), device=dev) for s in slots]
+    ys = [torch.empty((s.d_out, 1), device=dev) for s in slots]
+    xb = [x.to(torch.bfloat16).T.contiguous() for x in xs]
+    ws = torch.empty(max(4 * s.d_in for s in slots) + 64, dtype=torch.uint8, device=dev)
+
+    def fused():
+        for s, x, y in zip(slots, xs, ys):
+            q.decode_gemv(s.packed, s.row_norm, s.chan_scale, s.signs, s.sigma, mc.codebook, s.params, x, y, ws)
+
+    def bf16():
+        for s, x in zip(slots, xb):
+            torch.matmul(s.w_hat, x)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(calls):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / calls * 1e3  # microseconds per round
+
+    t_fused, t_bf16 = timed(fused), timed(bf16)
+    B = int(np.log2(mc.spec.K))
+    packed_bytes = sum(s.d_out * s.d_in * B / 16 for s in slots)
+    return {"matrices": [[s.d_out, s.d_in] for s in slots], "vectors": 1, "us_per_round": t_fused,
+            "packed_gb_s": packed_bytes / t_fused / 1e3, "frac_of_hbm_peak": packed_bytes / t_fused / 1e3 / peak_gbs,
+            "bf16_product_on_decoded_us": t_bf16, "kernel_launches_per_round": len(slots),
+            "note": "bound by the shared-memory gather of one codeword per pair, not by HBM"}
 
 
 def load_traffic_note():
