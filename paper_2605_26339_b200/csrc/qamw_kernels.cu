@@ -1000,6 +1000,96 @@ __host__ __device__ inline long long dist_item_count(int d_out, int d_in) {
     return (long long)((d_in + 8 * kDistThreads - 1) / (8 * kDistThreads)) * ((d_out + kDistRows - 1) / kDistRows);
 }
 
+// bf16 matrices in the 16-byte layout: the rows of a thread's work items form one stream that runs
+// through a private shared-memory ring of kDistDepth rows (two 16-byte asynchronous copies per row,
+// kDistDepth - 1 rows ahead, across item boundaries).  With the rows held in registers two rows were
+// in flight per thread and the kernel waited on memory latency; the ring keeps about 140 KB per SM in
+// flight without a register per byte.  A thread reads back only what it copied itself: no barrier.
+constexpr int kDistDepth = 8;
+struct DistCursor {
+    long long item;
+    int row, r1, j0;
+    bool valid;  // the thread's columns lie inside the matrix
+};
+__device__ __forceinline__ void dist_cursor_open(DistCursor& c, int d_out, int d_in, int col_tiles) {
+    const int chunk = int(c.item / col_tiles), tile = int(c.item - (long long)chunk * col_tiles);
+    c.j0 = (tile * kDistThreads + int(threadIdx.x)) * 8;
+    c.valid = c.j0 < d_in;
+    c.row = chunk * kDistRows;
+    c.r1 = min(d_out, c.row + kDistRows);
+}
+__device__ __forceinline__ void dist_items_stream(const __nv_bfloat16* W, long long w_row_stride, const __nv_bfloat16* What,
+                                                  const float* act_rms, int d_out, int d_in, long long first,
+                                                  long long last, long long step, double& s0, double& s1, double& s2,
+                                                  double& s3) {
+    __shared__ uint4 ring[kDistDepth][2][kDistThreads];
+    if (first >= last) return;
+    const int col_tiles = (d_in + 8 * kDistThreads - 1) / (8 * kDistThreads);
+    DistCursor prod, cons;
+    prod.item = cons.item = first;
+    dist_cursor_open(prod, d_out, d_in, col_tiles);
+    cons = prod;
+    int issued = 0;
+    auto issue = [&]() {  // one commit group per row of the stream, empty past its end
+        if (prod.item < last) {
+            if (prod.valid) {
+                cp_async(&ring[issued % kDistDepth][0][threadIdx.x], W + (long long)prod.row * w_row_stride + prod.j0, 4);
+                cp_async(&ring[issued % kDistDepth][1][threadIdx.x], What + (long long)prod.row * d_in + prod.j0, 4);
+            }
+            if (++prod.row == prod.r1) {
+                prod.item += step;
+                if (prod.item < last) dist_cursor_open(prod, d_out, d_in, col_tiles);
+            }
+        }
+        ++issued;
+        cp_async_commit();
+    };
+    for (int i = 0; i < kDistDepth - 1; ++i) issue();
+    double E[8], Q[8];
+    float rj[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) E[e] = Q[e] = 0.0;
+    bool fresh = true;
+    for (int taken = 0; cons.item < last; ++taken) {
+        if (fresh) {  // the activation weights of this item's columns, needed when the item ends
+#pragma unroll
+            for (int e = 0; e < 8; ++e) rj[e] = act_rms && cons.valid ? __ldg(act_rms + cons.j0 + e) : 1.0f;
+            fresh = false;
+        }
+        asm volatile("cp.async.wait_group %0;" ::"n"(kDistDepth - 2) : "memory");
+        const uint4 wv = ring[taken % kDistDepth][0][threadIdx.x], hv = ring[taken % kDistDepth][1][threadIdx.x];
+        issue();  // refills the slot read one row ago
+        if (cons.valid) {
+            const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w}, hw[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const double w0 = double(__uint_as_float(ww[i] << 16)), w1 = double(__uint_as_float(ww[i] & 0xffff0000u));
+                const double d0 = w0 - double(__uint_as_float(hw[i] << 16));
+                const double d1 = w1 - double(__uint_as_float(hw[i] & 0xffff0000u));
+                E[2 * i] = fma(d0, d0, E[2 * i]);
+                Q[2 * i] = fma(w0, w0, Q[2 * i]);
+                E[2 * i + 1] = fma(d1, d1, E[2 * i + 1]);
+                Q[2 * i + 1] = fma(w1, w1, Q[2 * i + 1]);
+            }
+        }
+        if (++cons.row == cons.r1) {  // end of the item: weight the column sums and start over
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const double r2 = double(rj[e]) * double(rj[e]);
+                s0 += E[e];
+                s1 += Q[e];
+                s2 = fma(r2, E[e], s2);
+                s3 = fma(r2, Q[e], s3);
+                E[e] = Q[e] = 0.0;
+            }
+            cons.item += step;
+            if (cons.item < last) dist_cursor_open(cons, d_out, d_in, col_tiles);
+            fresh = true;
+        }
+    }
+    cp_async_wait_all();
+}
+
 // The work items `first`, `first + step`, ... below `last` of one matrix, added into the thread's
 // four running sums.
 template <bool BF16>
@@ -1007,6 +1097,11 @@ __device__ __forceinline__ void dist_items(const void* W, long long w_row_stride
                                            const float* act_rms, int d_out, int d_in, int vec, long long first,
                                            long long last, long long step, double& s0, double& s1, double& s2,
                                            double& s3) {
+    if (BF16 && vec) {
+        dist_items_stream(static_cast<const __nv_bfloat16*>(W), w_row_stride, What, act_rms, d_out, d_in, first, last, step,
+                          s0, s1, s2, s3);
+        return;
+    }
     const int col_tiles = (d_in + 8 * kDistThreads - 1) / (8 * kDistThreads);
     for (long long item = first; item < last; item += step) {
         const int chunk = int(item / col_tiles), tile = int(item - (long long)chunk * col_tiles);
@@ -1017,46 +1112,6 @@ __device__ __forceinline__ void dist_items(const void* W, long long w_row_stride
 #pragma unroll
         for (int e = 0; e < 8; ++e) E[e] = Q[e] = 0.0;
         int row = r0;
-        if (BF16 && vec) {
-            // bf16 fast path: the next two rows are loaded (as raw 16-byte words) before the current two
-            // are converted and accumulated, so four rows of loads are in flight per thread
-            auto ld = [&](int rw, uint4& wv, uint4& hv) {
-                const __nv_bfloat16* wrow = reinterpret_cast<const __nv_bfloat16*>(W) + (long long)rw * w_row_stride;
-                wv = __ldg(reinterpret_cast<const uint4*>(wrow + j0));
-                hv = __ldg(reinterpret_cast<const uint4*>(What + (long long)rw * d_in + j0));
-            };
-            auto acc = [&](const uint4& wv, const uint4& hv) {
-                const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w}, hw[4] = {hv.x, hv.y, hv.z, hv.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const double w0 = double(__uint_as_float(ww[i] << 16)), w1 = double(__uint_as_float(ww[i] & 0xffff0000u));
-                    const double d0 = w0 - double(__uint_as_float(hw[i] << 16));
-                    const double d1 = w1 - double(__uint_as_float(hw[i] & 0xffff0000u));
-                    E[2 * i] = fma(d0, d0, E[2 * i]);
-                    Q[2 * i] = fma(w0, w0, Q[2 * i]);
-                    E[2 * i + 1] = fma(d1, d1, E[2 * i + 1]);
-                    Q[2 * i + 1] = fma(w1, w1, Q[2 * i + 1]);
-                }
-            };
-            uint4 cw[2], ch[2], nw[2], nh[2];
-            if (row + 2 <= r1) {
-                ld(row, cw[0], ch[0]);
-                ld(row + 1, cw[1], ch[1]);
-            }
-            for (; row + 2 <= r1; row += 2) {
-                const bool more = row + 4 <= r1;
-                if (more) {
-                    ld(row + 2, nw[0], nh[0]);
-                    ld(row + 3, nw[1], nh[1]);
-                }
-                acc(cw[0], ch[0]);
-                acc(cw[1], ch[1]);
-                if (more) {
-                    cw[0] = nw[0]; ch[0] = nh[0];
-                    cw[1] = nw[1]; ch[1] = nh[1];
-                }
-            }
-        }
         for (; row + 2 <= r1; row += 2) {  // generic path: two rows in flight per thread
             float w[2][8], h[2][8];
 #pragma unroll

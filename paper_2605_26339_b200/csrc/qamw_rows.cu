@@ -192,6 +192,12 @@ __device__ __forceinline__ int4 block_span(const int4* spans, int d_out_single) 
 // ---------------------------------------------------------------------------------------------
 // decoder
 // ---------------------------------------------------------------------------------------------
+constexpr int kDecodeDepth = 4;
+template <int N>
+__device__ __forceinline__ void cp_async_wait_pending() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
 struct Decode2Args {
     const MatDesc* descs;    // device array, or NULL: `one` is the only matrix
     MatDesc one;
@@ -203,8 +209,10 @@ struct Decode2Args {
     float inv_sqrt_b;
 };
 
-// A warp streams its segment of the packed row through its own two-deep shared-memory ring (16-byte
-// asynchronous copies); nothing is shared between warps after the prologue, so there is no barrier.
+// A warp streams its segment of the packed row through its own shared-memory ring of kDecodeDepth rows
+// (16-byte asynchronous copies, kDecodeDepth - 1 rows ahead: with one row in flight per warp the reads
+// are bound by memory latency); nothing is shared between warps after the prologue, so there is no
+// barrier.
 // Per row a thread reads its 4 NS B index bits as two runs of 32-bit words, gathers the codewords
 // (stored as (x + y, x - y): butterfly stage h = 1) from its own bank-separated copy, scales them by
 // the pair scales, runs the remaining butterflies and writes bf16.
@@ -219,12 +227,12 @@ __global__ void __launch_bounds__(NS == 4 ? 512 : 896, 1) decode2_kernel(const D
     const uint32_t mask = (1u << B) - 1u;
     const uint32_t cb_stride = 8u << a.log2c;
     const uint32_t cb = smem_addr(smem) + 8u * (threadIdx.x & ((1 << a.log2c) - 1));
-    unsigned char* stage = smem + ((size_t(a.K) * 8) << a.log2c) + size_t(warp) * 2 * a.stage_bytes;
+    unsigned char* stage = smem + ((size_t(a.K) * 8) << a.log2c) + size_t(warp) * kDecodeDepth * a.stage_bytes;
     const uint32_t stage_addr = smem_addr(stage);
 
     fill_codebook_copies(reinterpret_cast<float2*>(smem), a.codebook, a.K, a.log2c, true);
     // the 16 bytes after a staged segment are read (and masked away) by the last threads: keep them defined
-    if (lane < 8) reinterpret_cast<uint32_t*>(stage + (lane >> 2) * a.stage_bytes + a.seg_bytes)[lane & 3] = 0u;
+    if (lane < 4 * kDecodeDepth) reinterpret_cast<uint32_t*>(stage + (lane >> 2) * a.stage_bytes + a.seg_bytes)[lane & 3] = 0u;
     __syncthreads();
 
     // where this thread's index bits sit inside a staged segment: two runs (the lower and the upper
@@ -256,17 +264,21 @@ __global__ void __launch_bounds__(NS == 4 ? 512 : 896, 1) decode2_kernel(const D
         const int n_chunks = max(0, min(a.seg_bytes, row_bytes - int(seg_off))) >> 4;
         // at most 48 chunks of 16 bytes per segment: two predicated copies per lane, no loop
         const bool copy0 = lane < n_chunks, copy1 = lane + 32 < n_chunks;
-        auto issue_row = [&](const unsigned char* src, int buf) {
-            unsigned char* dst = stage + buf * a.stage_bytes;
-            if (copy0) cp_async(dst + (lane << 4), src + (lane << 4), 4);
-            if (copy1) cp_async(dst + ((lane + 32) << 4), src + ((lane + 32) << 4), 4);
-            cp_async_commit();
-        };
         const unsigned char* src = d.packed + (long long)row0 * pstride + seg_off;  // next row to fetch
         const long long src_step = (long long)row_step * pstride;
+        int issued = 0;
+        auto issue_row = [&]() {  // one commit group per row, empty past the end
+            if (issued < n_rows) {
+                unsigned char* dst = stage + (issued % kDecodeDepth) * a.stage_bytes;
+                if (copy0) cp_async(dst + (lane << 4), src + (lane << 4), 4);
+                if (copy1) cp_async(dst + ((lane + 32) << 4), src + ((lane + 32) << 4), 4);
+                src += src_step;
+            }
+            ++issued;
+            cp_async_commit();
+        };
         __syncwarp();  // the previous matrix's last row has been read by every lane
-        issue_row(src, 0);
-        src += src_step;
+        for (int i = 0; i < kDecodeDepth - 1; ++i) issue_row();
 
         // per-column constants of this warp's segment
         const int oct0 = seg * (WE / 8);  // first octet of the segment
@@ -299,16 +311,12 @@ __global__ void __launch_bounds__(NS == 4 ? 512 : 896, 1) decode2_kernel(const D
         const long long out_step = (long long)row_step * d_in;
         const float* rnp = d.row_norm + row0;
 
-        int buf = 0;
-        for (int it = 0; it < n_rows; ++it, buf ^= 1, orow += out_step, rnp += row_step) {
+        for (int it = 0; it < n_rows; ++it, orow += out_step, rnp += row_step) {
             const float rn = __ldg(rnp);
-            cp_async_wait_all();
-            __syncwarp();  // every lane's part of this row has landed; the other buffer is no longer read
-            if (it + 1 < n_rows) {
-                issue_row(src, buf ^ 1);
-                src += src_step;
-            }
-            const uint32_t in = stage_addr + uint32_t(buf * a.stage_bytes);
+            cp_async_wait_pending<kDecodeDepth - 2>();
+            __syncwarp();  // every lane's part of this row has landed; the buffer refilled next is no longer read
+            issue_row();
+            const uint32_t in = stage_addr + uint32_t((it % kDecodeDepth) * a.stage_bytes);
             f32x2 P[NS][4];
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
@@ -927,7 +935,7 @@ int rows_decode(const MatDesc* descs_dev, const MatDesc* descs_host, int n, cons
     a.seg_bytes = 16 * NS * a.log2K;
     a.stage_bytes = (a.seg_bytes + 16 + 127) & ~127;  // 128-byte aligned ring buffers
     a.inv_sqrt_b = float(1.0 / std::sqrt(double(block)));
-    const size_t stage_total = size_t(kWarps) * 2 * a.stage_bytes;
+    const size_t stage_total = size_t(kWarps) * kDecodeDepth * a.stage_bytes;
     a.log2c = pick_copies(K, std::min(size_t(128) * 1024, kSmemLimit - stage_total));
     const size_t smem = (size_t(K) * 8 << a.log2c) + stage_total;
     int grid = sm_count();
