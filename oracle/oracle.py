@@ -302,6 +302,20 @@ def train_codebook(K, n_samples=1 << 20, seed=0, max_iters=100, rel_tol=1e-6, wa
     return cb, mse.value, iters.value
 
 
+def train_codebook_on(samples, K, max_iters=100, rel_tol=1e-6):
+    """The trainer's iteration on a given [n, 2] float64 sample array -> (codebook f32, mse, updates, trace)."""
+    s = _c(samples, np.float64)
+    cb = np.empty((K, 2), np.float32)
+    mse = C.c_double()
+    iters = C.c_int()
+    trace = np.full(max_iters + 2, np.nan, np.float64)
+    rc = lib().orc_train_codebook_on(_p(s), C.c_uint64(s.shape[0]), C.c_int(K), C.c_int(max_iters), C.c_double(rel_tol),
+                                     _p(cb), C.byref(mse), C.byref(iters), _p(trace))
+    if rc != ORC_OK:
+        raise ValueError(f"orc_train_codebook_on failed: {rc}")
+    return cb, mse.value, iters.value, trace[~np.isnan(trace)]
+
+
 def codebook_mse(codebook, n_samples, seed) -> float:
     cb = _c(codebook, np.float32)
     return float(lib().orc_codebook_mse(_p(cb), C.c_int(cb.shape[0]), C.c_uint64(n_samples), C.c_uint64(seed)))

@@ -607,15 +607,28 @@ static int cmp_codeword(const void *pa, const void *pb) {
  * mse_out = mean squared distance of the samples to the final f32 codebook;
  * mse_trace (optional, max_iters+1 doubles) receives D_1, D_2, ...
  */
+/* The same iteration on a sample array handed in (n pairs of doubles): what a codebook fitted to a
+ * matrix's own pairs uses. */
+int orc_train_codebook_on(const double *samples, uint64_t n, int K, int max_iters, double rel_tol,
+                          float *codebook_out, double *mse_out, int *iters_out, double *mse_trace);
+
 int orc_train_codebook(int K, uint64_t n, uint64_t seed, int max_iters, double rel_tol,
                        float *codebook_out, double *mse_out, int *iters_out, double *mse_trace) {
     if (K < 1 || n < (uint64_t)K || max_iters < 0) return ORC_ERR_ARG;
     double *samples = (double *)malloc(sizeof(double) * 2 * n);
+    orc_gauss_pairs(seed, n, samples);
+    const int rc = orc_train_codebook_on(samples, n, K, max_iters, rel_tol, codebook_out, mse_out, iters_out, mse_trace);
+    free(samples);
+    return rc;
+}
+
+int orc_train_codebook_on(const double *samples, uint64_t n, int K, int max_iters, double rel_tol,
+                          float *codebook_out, double *mse_out, int *iters_out, double *mse_trace) {
+    if (!samples || K < 1 || n < (uint64_t)K || max_iters < 0) return ORC_ERR_ARG;
     double *cb = (double *)malloc(sizeof(double) * 2 * (size_t)K);
     double *sum = (double *)malloc(sizeof(double) * 2 * (size_t)K);
     int64_t *cnt = (int64_t *)malloc(sizeof(int64_t) * (size_t)K);
     int32_t *assign = (int32_t *)malloc(sizeof(int32_t) * n);
-    orc_gauss_pairs(seed, n, samples);
     const double root2 = 1.4142135623730950488016887242097;
     for (int c = 0; c < 2 * K; ++c) cb[c] = root2 * samples[c];
     double prev = INFINITY;
@@ -648,7 +661,6 @@ int orc_train_codebook(int K, uint64_t n, uint64_t seed, int max_iters, double r
         *mse_out = orc_lloyd_assign(samples, n, cb, K, NULL);
     }
     if (iters_out) *iters_out = updates;
-    free(samples);
     free(cb);
     free(sum);
     free(cnt);

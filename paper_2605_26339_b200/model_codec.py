@@ -70,6 +70,37 @@ def choose_alpha(W: torch.Tensor, act_rms: torch.Tensor, codebook: q.Codebook, b
     return best, scores
 
 
+def fit_codebook(W: torch.Tensor, act_rms: Optional[torch.Tensor], alpha: float, block: int, K: int,
+                 n_pairs: int = 1 << 20, max_iters: int = 100, rel_tol: float = 1e-6,
+                 sign_seed: int = q.DEFAULT_SIGN_SEED, seed: int = 0):
+    """Codebook fitted to one matrix's own pairs instead of the unit circular Gaussian (the per-checkpoint
+    codebook the paper names as follow-up work, Section 3.6 / Limitations): the rows go through channel
+    scaling, normalisation and rotation (qamw_rotate), the pairs are divided by the calibrated pair
+    scales, and the device trainer runs Lloyd iterations on up to n_pairs of them (rows taken at a fixed
+    stride).  Returns dict(codebook, mse, iters, seconds, sigma, rows)."""
+    dev = W.device
+    d_out, d_in = W.shape
+    p = q.make_params(W, d_out, d_in, block, K)
+    signs = torch.from_numpy(q.make_signs(sign_seed, d_in)).to(dev)
+    s = None
+    if alpha and act_rms is not None:
+        s = torch.from_numpy(q.channel_scales(act_rms.detach().cpu().numpy(), alpha)).to(dev)
+    sigma = torch.empty(d_in // 2, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(8, q.calibrate_workspace_bytes(p)), dtype=torch.uint8, device=dev)
+    q.calibrate(W, p, s, signs, sigma, ws)
+    n_rows = max(1, min(d_out, (n_pairs + d_in // 2 - 1) // (d_in // 2)))
+    rows = torch.div(torch.arange(n_rows, device=dev) * d_out, n_rows, rounding_mode="floor")
+    Wsub = W.index_select(0, rows).contiguous()
+    ps = q.make_params(Wsub, n_rows, d_in, block, K)
+    y = torch.empty((n_rows, d_in), dtype=torch.float32, device=dev)
+    norm = torch.empty(n_rows, dtype=torch.float32, device=dev)
+    q.rotate(Wsub, ps, s, signs, y, norm)
+    z = (y.view(n_rows, d_in // 2, 2) / sigma[None, :, None]).reshape(-1, 2)[:n_pairs].double().contiguous()
+    out = q.train_codebook_gpu(K, max_iters=max_iters, rel_tol=rel_tol, samples=z, seed=seed)
+    out.update(sigma=sigma, rows=n_rows)
+    return out
+
+
 @dataclass
 class MatrixSlot:
     """Device-resident state of one weight matrix."""

@@ -62,3 +62,27 @@ def test_device_generated_samples_give_the_golden_codebook_quality(orc):
     print(f"LLOYD K={K}: device {out['seconds']:.3f} s, {out['iters']} updates")
     again = q.train_codebook_gpu(K, 1 << 20, 0, 100, 1e-6)
     assert np.array_equal(again["codebook"], out["codebook"])  # reproducible run to run
+
+
+def test_codebook_fitted_to_a_matrix_beats_the_gaussian_one_on_it(orc):
+    """Per-matrix codebook (Lloyd on the matrix's own rotated, scaled pairs): its quantisation error on
+    those pairs is not above the Gaussian-trained codebook's, and the device trainer's result on the
+    pairs equals the oracle trainer's."""
+    from paper_2605_26339_b200.model_codec import fit_codebook
+    g = torch.Generator().manual_seed(12)
+    d_out, d_in, K = 512, 1024, 64
+    # light-tailed rows (uniform entries): after a block-32 rotation the pairs are visibly non-Gaussian
+    W = ((torch.rand((d_out, d_in), generator=g) - 0.5) * torch.exp(0.5 * torch.randn((d_out, 1), generator=g))).to(DEV)
+    fit = fit_codebook(W, None, 0.0, 2, K, n_pairs=1 << 16, max_iters=40, rel_tol=1e-7)
+    assert fit["codebook"].shape == (K, 2) and np.isfinite(fit["codebook"]).all()
+    # the same pairs through the oracle: same codebook
+    rows = (np.arange(fit["rows"]) * d_out) // fit["rows"]
+    signs = q.make_signs(q.DEFAULT_SIGN_SEED, d_in)
+    Wh = W.cpu().numpy()
+    y = np.stack([orc.front_row(Wh[r], 2, None, signs)[0] for r in rows])
+    z = (y.reshape(len(rows), d_in // 2, 2) / fit["sigma"].cpu().numpy()[None, :, None]).reshape(-1, 2)[: 1 << 16]
+    ref_cb, ref_mse, _, _ = orc.train_codebook_on(z.astype(np.float64), K, 40, 1e-7)
+    assert np.array_equal(fit["codebook"], ref_cb)
+    gauss = load_golden_codebook(K)
+    _, mse_gauss = orc.lloyd_assign(z.astype(np.float64), gauss.astype(np.float64))
+    assert fit["mse"] < mse_gauss
