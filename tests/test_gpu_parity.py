@@ -580,3 +580,35 @@ def test_one_call_quantize_equals_the_separate_calls(orc):
     q.calibrate(Wd, p, None, signs_out, sigma_out, ws, st)
     q.encode(Wd, p, None, signs_out, sigma_out, c.cb, packed2, norm2)
     assert torch.equal(packed, packed2) and torch.equal(norm, norm2)
+
+
+@pytest.mark.parametrize("d_out,d_in", [(1, 8), (15, 1000), (16, 1024), (17, 2056), (100, 3072), (33, 8200)])
+def test_distortion_sums_for_short_and_ragged_streams(orc, d_out, d_in):
+    """The four sums of the distortion reduction (Corollaries 3 and 4) on bf16 pairs (W, W_hat) whose row
+    streams are shorter than, equal to and longer than the copy ring, with columns that fill a thread
+    tile only partly: single-matrix call and one batch of three copies against the oracle."""
+    g = torch.Generator().manual_seed(d_out * 7919 + d_in)
+    W = (torch.randn((d_out, d_in), generator=g) * torch.exp(torch.randn((d_out, 1), generator=g))).to(torch.bfloat16)
+    What = (W.float() * (1 + 0.05 * torch.randn((d_out, d_in), generator=g))).to(torch.bfloat16)
+    What[0, 0] = 0.0
+    act = torch.exp(torch.randn(d_in, generator=g))
+    ref = orc.distortion(_to_bits(W), _to_bits(What), act.numpy())
+    Wd, Hd, ad = W.to(DEV), What.to(DEV), act.to(DEV)
+    p = q.make_params(Wd, d_out, d_in, 2, 64)
+    out4 = torch.full((4,), float("nan"), dtype=torch.float64, device=DEV)
+    q.distortion(Wd, Hd, ad, p, out4)
+    np.testing.assert_allclose(out4.cpu().numpy(), ref, rtol=1e-9)
+    ref_plain = orc.distortion(_to_bits(W), _to_bits(What), None)
+    q.distortion(Wd, Hd, None, p, out4)
+    np.testing.assert_allclose(out4.cpu().numpy(), ref_plain, rtol=1e-9)
+    # three matrices behind one batch handle: every one gets its own sums
+    cb = _codebook(orc, 64)[1]
+    dummy_b = torch.zeros(d_out * p.packed_row_stride + 64, dtype=torch.uint8, device=DEV)
+    dummy_f = torch.ones(max(d_out, d_in), dtype=torch.float32, device=DEV)
+    signs = torch.ones(d_in, dtype=torch.int8, device=DEV)
+    dists = [torch.full((4,), float("nan"), dtype=torch.float64, device=DEV) for _ in range(3)]
+    mats = [q.make_matrix(p, Wd, None, signs, dummy_f, ad, dummy_b, dummy_f, Hd, d) for d in dists]
+    batch = q.Batch(mats, cb)
+    batch.distortion()
+    for d in dists:
+        np.testing.assert_allclose(d.cpu().numpy(), ref, rtol=1e-9)
