@@ -1150,8 +1150,9 @@ __device__ __forceinline__ void dist_items(const void* W, long long w_row_stride
     }
 }
 
-// Block-wide sums of the four values (fixed order inside the block), added to out4 by four threads.
-__device__ __forceinline__ void dist_flush(double s0, double s1, double s2, double s3, double* out4) {
+// Block-wide sums of the four values (fixed order inside the block), added to out4 by four threads,
+// or stored there when the caller adds the blocks up itself.
+__device__ __forceinline__ void dist_flush(double s0, double s1, double s2, double s3, double* out4, bool store = false) {
     __shared__ double sh[4][kDistThreads / 32];
     s0 = warp_sum(s0); s1 = warp_sum(s1); s2 = warp_sum(s2); s3 = warp_sum(s3);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1161,7 +1162,8 @@ __device__ __forceinline__ void dist_flush(double s0, double s1, double s2, doub
     if (threadIdx.x < 4) {
         double v = 0;
         for (int w = 0; w < kDistThreads / 32; ++w) v += sh[threadIdx.x][w];
-        atomicAdd(out4 + threadIdx.x, v);
+        if (store) out4[threadIdx.x] = v;
+        else atomicAdd(out4 + threadIdx.x, v);
     }
 }
 
@@ -1175,28 +1177,43 @@ __global__ void __launch_bounds__(kDistThreads, 5) distortion_kernel(const void*
     dist_flush(s0, s1, s2, s3, out4);
 }
 
-// All matrices of a batch: block b owns a contiguous span of the concatenated item list.
+// All matrices of a batch: block b owns a contiguous span of the concatenated item list and leaves one
+// record of four partial sums per matrix of its span.  The block that finishes last (a ticket counter
+// behind a fence) adds the records of every matrix in block order and writes the matrix's four sums:
+// one launch, no atomics on the sums, the same bits on every run.
 template <bool BF16>
-__global__ void __launch_bounds__(kDistThreads, 5) distortion_batch_kernel(const MatDesc* descs, const int4* spans) {
+__global__ void __launch_bounds__(kDistThreads, 5) distortion_batch_kernel(const MatDesc* descs, const int4* spans,
+                                                                        const DistReduce red, int n_mats) {
     const int4 span = spans[blockIdx.x];
-    for (int m = span.x; m <= span.z; ++m) {
+    double* rec = red.partial + 4 * size_t(red.rec_off[blockIdx.x]);
+    for (int m = span.x; m <= span.z; ++m, rec += 4) {
         const MatDesc& d = descs[m];
         const long long first = m == span.x ? span.y : 0;
         const long long last = m == span.z ? span.w : dist_item_count(d.d_out, d.d_in);
-        if (first >= last) continue;
         const size_t esz = BF16 ? 2 : 4;
         const int vec = (d.d_in % 8 == 0) && (reinterpret_cast<uintptr_t>(d.W) % 16 == 0) &&
                         ((size_t(d.w_row_stride) * esz) % 16 == 0) && (reinterpret_cast<uintptr_t>(d.w_hat) % 16 == 0);
         double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
-        dist_items<BF16>(d.W, d.w_row_stride, static_cast<const __nv_bfloat16*>(d.w_hat), d.act_rms, d.d_out, d.d_in, vec,
-                         first, last, 1, s0, s1, s2, s3);
-        dist_flush(s0, s1, s2, s3, d.dist4);
+        if (first < last)
+            dist_items<BF16>(d.W, d.w_row_stride, static_cast<const __nv_bfloat16*>(d.w_hat), d.act_rms, d.d_out, d.d_in, vec,
+                             first, last, 1, s0, s1, s2, s3);
+        dist_flush(s0, s1, s2, s3, rec, true);
     }
-}
-
-__global__ void zero_dist_kernel(const MatDesc* descs, int n) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < 4 * n) descs[i >> 2].dist4[i & 3] = 0.0;
+    __shared__ bool last_block;
+    __threadfence();  // this block's records are visible before its ticket is
+    __syncthreads();
+    if (threadIdx.x == 0) last_block = atomicAdd(red.counter, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!last_block) return;
+    __threadfence();
+    for (int idx = threadIdx.x; idx < 4 * n_mats; idx += blockDim.x) {
+        const int m = idx >> 2, t = idx & 3;
+        const BlockRange own = red.owner[m];
+        double v = 0.0;
+        for (int b = own.x; b <= own.y; ++b) v += __ldcg(red.partial + 4 * size_t(red.rec_off[b] + m - spans[b].x) + t);
+        descs[m].dist4[t] = v;
+    }
+    if (threadIdx.x == 0) *red.counter = 0u;  // ready for the next launch
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1311,11 +1328,11 @@ int launch_decode(const DecodeArgs& a, int blocks, size_t smem, cudaStream_t st)
 namespace qamw {
 int check_matrix_params(const qamw_params* p) { return check_params(p); }
 long long distortion_items(int d_out, int d_in) { return dist_item_count(d_out, d_in); }
-int distortion_batch_launch(const MatDesc* descs_dev, int n, const void* spans_dev, int blocks, int w_bf16, void* stream) {
+int distortion_batch_launch(const MatDesc* descs_dev, int n, const void* spans_dev, int blocks, int w_bf16,
+                            const DistReduce& red, void* stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    zero_dist_kernel<<<(4 * n + 255) / 256, 256, 0, st>>>(descs_dev, n);
-    if (w_bf16) distortion_batch_kernel<true><<<blocks, kDistThreads, 0, st>>>(descs_dev, static_cast<const int4*>(spans_dev));
-    else distortion_batch_kernel<false><<<blocks, kDistThreads, 0, st>>>(descs_dev, static_cast<const int4*>(spans_dev));
+    if (w_bf16) distortion_batch_kernel<true><<<blocks, kDistThreads, 0, st>>>(descs_dev, static_cast<const int4*>(spans_dev), red, n);
+    else distortion_batch_kernel<false><<<blocks, kDistThreads, 0, st>>>(descs_dev, static_cast<const int4*>(spans_dev), red, n);
     return finish_launch("distortion_batch_kernel");
 }
 }  // namespace qamw

@@ -1078,6 +1078,12 @@ struct qamw_batch {
     RowSet enc[3];                  // encoder: one set per block size (20, 24, 28 warps)
     int4* d_spans_dist = nullptr;   // distortion: spans of the concatenated work-item list, over dec.d_descs
     int n_blocks_dist = 0;
+    double* d_dist_partial = nullptr;   // one record of four sums per (block, matrix of its span)
+    int* d_dist_rec_off = nullptr;      // first record of every block
+    BlockRange* d_dist_owner = nullptr;       // per matrix: first and last block whose span holds it
+    unsigned int* d_dist_counter = nullptr;  // ticket of the blocks; zero between launches
+    MatDesc* d_cal_all = nullptr;       // calibration descriptors of all block-size classes, for the one finish launch
+    int cal_all_n = 0, cal_all_max_pairs = 0;
     RowSet cal[3];                  // calibration: the encoder's sets again, spans over the calibration rows
     size_t cal_bytes = 0;           // partial-sum slots of all matrices (front of the caller's workspace)
     std::vector<size_t> ws_offset;  // calibration scratch of item i inside the caller's workspace
@@ -1200,6 +1206,16 @@ extern "C" int qamw_batch_create(const qamw_matrix* items, int n, const qamw_cod
         if (e == cudaSuccess) e = cudaMalloc(&r.d_spans, sizeof(int4) * spans.size());
         if (e == cudaSuccess) e = cudaMemcpy(r.d_spans, spans.data(), sizeof(int4) * spans.size(), cudaMemcpyHostToDevice);
     }
+    if (e == cudaSuccess) {  // all calibration descriptors in one array: one finish launch for every class
+        std::vector<MatDesc> all;
+        for (int c = 0; c < 3; ++c) all.insert(all.end(), b->cal[c].descs.begin(), b->cal[c].descs.end());
+        b->cal_all_n = int(all.size());
+        for (const MatDesc& d : all) b->cal_all_max_pairs = std::max(b->cal_all_max_pairs, d.d_in / 2);
+        if (!all.empty()) {
+            e = cudaMalloc(&b->d_cal_all, sizeof(MatDesc) * all.size());
+            if (e == cudaSuccess) e = cudaMemcpy(b->d_cal_all, all.data(), sizeof(MatDesc) * all.size(), cudaMemcpyHostToDevice);
+        }
+    }
     if (e == cudaSuccess) {  // distortion: equal numbers of work items per block, sixteen blocks per SM
         std::vector<MatDesc> items_as_rows(b->dec.descs);
         std::vector<int> unit(size_t(n), 1);
@@ -1213,6 +1229,23 @@ extern "C" int qamw_batch_create(const qamw_matrix* items, int n, const qamw_cod
         make_spans(items_as_rows.data(), n, b->n_blocks_dist, unit.data(), &spans);
         e = cudaMalloc(&b->d_spans_dist, sizeof(int4) * spans.size());
         if (e == cudaSuccess) e = cudaMemcpy(b->d_spans_dist, spans.data(), sizeof(int4) * spans.size(), cudaMemcpyHostToDevice);
+        // records of the blocks' partial sums and, per matrix, the blocks that own a piece of it
+        std::vector<int> rec_off(spans.size() + 1, 0);
+        std::vector<BlockRange> owner(size_t(n), BlockRange{int(spans.size()), -1});
+        for (size_t k = 0; k < spans.size(); ++k) {
+            rec_off[k + 1] = rec_off[k] + (spans[k].z - spans[k].x + 1);
+            for (int i = spans[k].x; i <= spans[k].z; ++i) {
+                owner[size_t(i)].x = std::min(owner[size_t(i)].x, int(k));
+                owner[size_t(i)].y = std::max(owner[size_t(i)].y, int(k));
+            }
+        }
+        if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_partial, sizeof(double) * 4 * size_t(std::max(1, rec_off.back())));
+        if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_rec_off, sizeof(int) * rec_off.size());
+        if (e == cudaSuccess) e = cudaMemcpy(b->d_dist_rec_off, rec_off.data(), sizeof(int) * rec_off.size(), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_owner, sizeof(BlockRange) * size_t(n));
+        if (e == cudaSuccess) e = cudaMemcpy(b->d_dist_owner, owner.data(), sizeof(BlockRange) * size_t(n), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_counter, sizeof(unsigned int));
+        if (e == cudaSuccess) e = cudaMemset(b->d_dist_counter, 0, sizeof(unsigned int));
     }
     if (e != cudaSuccess) {
         set_cuda_error("qamw_batch_create", int(e));
@@ -1231,6 +1264,11 @@ extern "C" void qamw_batch_destroy(qamw_batch* b) {
         free_row_set(b->cal[c]);
     }
     if (b->d_spans_dist) cudaFree(b->d_spans_dist);
+    if (b->d_dist_partial) cudaFree(b->d_dist_partial);
+    if (b->d_dist_rec_off) cudaFree(b->d_dist_rec_off);
+    if (b->d_dist_owner) cudaFree(b->d_dist_owner);
+    if (b->d_dist_counter) cudaFree(b->d_dist_counter);
+    if (b->d_cal_all) cudaFree(b->d_cal_all);
     delete b;
 }
 
@@ -1249,7 +1287,10 @@ extern "C" int qamw_calibrate_batch(const qamw_batch* b, void* workspace, size_t
     const uint32_t flags = b->items[0].p.flags;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     bool zeroed = false;
-    for (int c = 0; c < 3; ++c) {  // one pass and one finish launch per block size
+    // One pass per block size; the partial sums of all of them are finished by one launch, unless a class
+    // had to go through the single-matrix kernels (then the classes that did not are finished one by one).
+    bool fast[3] = {false, false, false}, any_general = false;
+    for (int c = 0; c < 3; ++c) {
         const RowSet& set = b->cal[c];
         if (set.descs.empty()) continue;
         int rc = QAMW_ERR_SHAPE;
@@ -1264,15 +1305,10 @@ extern "C" int qamw_calibrate_batch(const qamw_batch* b, void* workspace, size_t
             }
             rc = rows_encode(set.d_descs, set.descs.data(), int(set.descs.size()), set.d_spans, b->n_blocks, b->block, b->K,
                              b->w_dtype == QAMW_DTYPE_BF16, nullptr, flags, status_out, stream, ws);
-            if (rc == QAMW_OK) {
-                int max_pairs = 0;
-                for (const MatDesc& d : set.descs) max_pairs = std::max(max_pairs, d.d_in / 2);
-                calibrate_finish2_kernel<<<dim3(unsigned((max_pairs + 31) / 32), unsigned(set.descs.size())),
-                                           32 * kFinishSlices, 0, st>>>(set.d_descs, ws);
-                rc = launch_check("calibrate_finish2_kernel");
-            }
+            fast[c] = rc == QAMW_OK;
         }
         if (rc == QAMW_ERR_SHAPE) {  // some matrix of the set needs the general kernel: one call per matrix
+            any_general = true;
             rc = QAMW_OK;
             for (size_t k = 0; k < set.index.size() && rc == QAMW_OK; ++k) {
                 const int i = set.index[k];
@@ -1281,6 +1317,21 @@ extern "C" int qamw_calibrate_batch(const qamw_batch* b, void* workspace, size_t
                                     workspace_bytes - b->cal_bytes - b->ws_offset[i], status_out, stream);
             }
         }
+        if (rc) return rc;
+    }
+    if (!any_general && (fast[0] || fast[1] || fast[2])) {
+        calibrate_finish2_kernel<<<dim3(unsigned((b->cal_all_max_pairs + 31) / 32), unsigned(b->cal_all_n)), 32 * kFinishSlices, 0,
+                                   st>>>(b->d_cal_all, ws);
+        return launch_check("calibrate_finish2_kernel");
+    }
+    for (int c = 0; c < 3; ++c) {
+        if (!fast[c]) continue;
+        const RowSet& set = b->cal[c];
+        int max_pairs = 0;
+        for (const MatDesc& d : set.descs) max_pairs = std::max(max_pairs, d.d_in / 2);
+        calibrate_finish2_kernel<<<dim3(unsigned((max_pairs + 31) / 32), unsigned(set.descs.size())), 32 * kFinishSlices, 0,
+                                   st>>>(set.d_descs, ws);
+        const int rc = launch_check("calibrate_finish2_kernel");
         if (rc) return rc;
     }
     return QAMW_OK;
@@ -1339,6 +1390,11 @@ extern "C" int qamw_distortion_batch(const qamw_batch* b, void* stream) {
         const qamw_matrix& it = b->items[i];
         if (!it.W || !it.w_hat_bf16 || !it.dist4) return QAMW_ERR_ARG;
     }
+    DistReduce red;
+    red.partial = b->d_dist_partial;
+    red.rec_off = b->d_dist_rec_off;
+    red.owner = b->d_dist_owner;
+    red.counter = b->d_dist_counter;
     return distortion_batch_launch(b->dec.d_descs, b->n, b->d_spans_dist, b->n_blocks_dist, b->w_dtype == QAMW_DTYPE_BF16,
-                                   stream);
+                                   red, stream);
 }

@@ -257,10 +257,10 @@ class ModelCodec:
         # class of row lengths (rows of up to 11264 elements, longer rows)
         n = len(self.slots)
         if self.use_batch and self.batch is not None:
-            # one encoder block size per class of row lengths; calibration = one pass and one finish launch
-            # per class; distortion = a zeroing launch and the batch kernel; one decode launch
+            # one encoder block size per class of row lengths: a calibration pass and an encode launch per
+            # class; one finish launch, one decode launch, one distortion launch
             classes = len({self._encoder_class(s.d_in) for s in self.slots})
-            return 2 * classes + classes + 1 + 2
+            return 2 * classes + 3
         return 5 * n
 
     @staticmethod

@@ -474,6 +474,12 @@ def test_batch_equals_single_matrix_calls(orc, shapes, block):
         assert torch.equal(x["packed"], y["packed"]) and torch.equal(x["norm"], y["norm"])
         assert torch.equal(x["what"].view(torch.int16), y["what"].view(torch.int16))
         np.testing.assert_allclose(x["dist"].cpu().numpy(), y["dist"].cpu().numpy(), rtol=1e-9)
+    # the batched sums are added in a fixed order: a second launch gives the same bits
+    first = [y["dist"].clone() for y in b]
+    batch.distortion()
+    torch.cuda.synchronize()
+    for f, y in zip(first, b):
+        assert torch.equal(f, y["dist"])
     # and the first matrix against the oracle, through the batch's outputs
     s0 = b[0]
     Wb = _to_bits(s0["W"])
