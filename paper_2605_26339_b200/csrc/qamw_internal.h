@@ -109,18 +109,18 @@ int sm_count();
 int check_matrix_params(const qamw_params* p);
 long long distortion_items(int d_out, int d_in);  // work items of the distortion kernel for one matrix
 // zeroes every matrix's four sums, then one launch over all matrices (spans of the concatenated item list)
-// Where the blocks of the batched distortion kernel leave their partial sums, and what the last block to
-// finish needs to add them up in a fixed order: records of four doubles, block b's first one at
-// rec_off[b] (one per matrix of its span); matrix m appears in the spans of blocks owner[m].x ..
-// owner[m].y; counter starts at zero and is reset by the last block.
-struct BlockRange {
-    int x, y;  // first and last block
+// Where the blocks of the batched distortion kernel leave their partial sums: records of four doubles,
+// matrix by matrix; matrix m appears in the spans of blocks owner[m].first .. owner[m].last and block b's
+// record for it is number owner[m].offset + b - owner[m].first.  counter is the ticket of the blocks;
+// the one that finishes last adds the records up in a fixed order and resets it.
+struct DistOwner {
+    int first, last;  // blocks
+    int offset;       // first record of the matrix
 };
 struct DistReduce {
     double* partial;
-    const int* rec_off;
-    const BlockRange* owner;
-    unsigned int* counter;
+    const DistOwner* owner;
+    unsigned int* counter;  // zero between launches
 };
 int distortion_batch_launch(const MatDesc* descs_dev, int n, const void* spans_dev, int blocks, int w_bf16,
                             const DistReduce& red, void* stream);  // QAMW_OK or the error code every entry point reports

@@ -1178,15 +1178,17 @@ __global__ void __launch_bounds__(kDistThreads, 5) distortion_kernel(const void*
 }
 
 // All matrices of a batch: block b owns a contiguous span of the concatenated item list and leaves one
-// record of four partial sums per matrix of its span.  The block that finishes last (a ticket counter
-// behind a fence) adds the records of every matrix in block order and writes the matrix's four sums:
-// one launch, no atomics on the sums, the same bits on every run.
+// record of four partial sums per matrix of its span.  The block that finishes last (one ticket counter
+// behind a fence) adds the records of every matrix in a fixed order -- a thread per sum for the matrices
+// a few blocks worked on, a warp per sum (lanes take every 32nd record, then a fixed tree) for a matrix
+// spread over many -- and writes the four sums: one launch, no atomics on the sums, the same bits on
+// every run.
+constexpr int kDistWideRecords = 64;
 template <bool BF16>
 __global__ void __launch_bounds__(kDistThreads, 5) distortion_batch_kernel(const MatDesc* descs, const int4* spans,
                                                                         const DistReduce red, int n_mats) {
     const int4 span = spans[blockIdx.x];
-    double* rec = red.partial + 4 * size_t(red.rec_off[blockIdx.x]);
-    for (int m = span.x; m <= span.z; ++m, rec += 4) {
+    for (int m = span.x; m <= span.z; ++m) {
         const MatDesc& d = descs[m];
         const long long first = m == span.x ? span.y : 0;
         const long long last = m == span.z ? span.w : dist_item_count(d.d_out, d.d_in);
@@ -1197,7 +1199,8 @@ __global__ void __launch_bounds__(kDistThreads, 5) distortion_batch_kernel(const
         if (first < last)
             dist_items<BF16>(d.W, d.w_row_stride, static_cast<const __nv_bfloat16*>(d.w_hat), d.act_rms, d.d_out, d.d_in, vec,
                              first, last, 1, s0, s1, s2, s3);
-        dist_flush(s0, s1, s2, s3, rec, true);
+        const DistOwner own = red.owner[m];
+        dist_flush(s0, s1, s2, s3, red.partial + 4 * size_t(own.offset + int(blockIdx.x) - own.first), true);
     }
     __shared__ bool last_block;
     __threadfence();  // this block's records are visible before its ticket is
@@ -1208,10 +1211,25 @@ __global__ void __launch_bounds__(kDistThreads, 5) distortion_batch_kernel(const
     __threadfence();
     for (int idx = threadIdx.x; idx < 4 * n_mats; idx += blockDim.x) {
         const int m = idx >> 2, t = idx & 3;
-        const BlockRange own = red.owner[m];
+        const DistOwner own = red.owner[m];
+        const int n_rec = own.last - own.first + 1;
+        if (n_rec > kDistWideRecords) continue;
+        const double* rec = red.partial + 4 * size_t(own.offset) + t;
         double v = 0.0;
-        for (int b = own.x; b <= own.y; ++b) v += __ldcg(red.partial + 4 * size_t(red.rec_off[b] + m - spans[b].x) + t);
+        for (int r = 0; r < n_rec; ++r) v += __ldcg(rec + 4 * size_t(r));
         descs[m].dist4[t] = v;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int idx = warp; idx < 4 * n_mats; idx += kDistThreads / 32) {
+        const int m = idx >> 2, t = idx & 3;
+        const DistOwner own = red.owner[m];
+        const int n_rec = own.last - own.first + 1;
+        if (n_rec <= kDistWideRecords) continue;
+        const double* rec = red.partial + 4 * size_t(own.offset) + t;
+        double v = 0.0;
+        for (int r = lane; r < n_rec; r += 32) v += __ldcg(rec + 4 * size_t(r));
+        v = warp_sum(v);
+        if (lane == 0) descs[m].dist4[t] = v;
     }
     if (threadIdx.x == 0) *red.counter = 0u;  // ready for the next launch
 }

@@ -1079,8 +1079,7 @@ struct qamw_batch {
     int4* d_spans_dist = nullptr;   // distortion: spans of the concatenated work-item list, over dec.d_descs
     int n_blocks_dist = 0;
     double* d_dist_partial = nullptr;   // one record of four sums per (block, matrix of its span)
-    int* d_dist_rec_off = nullptr;      // first record of every block
-    BlockRange* d_dist_owner = nullptr;       // per matrix: first and last block whose span holds it
+    DistOwner* d_dist_owner = nullptr;  // per matrix: first and last block whose span holds it, first record
     unsigned int* d_dist_counter = nullptr;  // ticket of the blocks; zero between launches
     MatDesc* d_cal_all = nullptr;       // calibration descriptors of all block-size classes, for the one finish launch
     int cal_all_n = 0, cal_all_max_pairs = 0;
@@ -1229,21 +1228,21 @@ extern "C" int qamw_batch_create(const qamw_matrix* items, int n, const qamw_cod
         make_spans(items_as_rows.data(), n, b->n_blocks_dist, unit.data(), &spans);
         e = cudaMalloc(&b->d_spans_dist, sizeof(int4) * spans.size());
         if (e == cudaSuccess) e = cudaMemcpy(b->d_spans_dist, spans.data(), sizeof(int4) * spans.size(), cudaMemcpyHostToDevice);
-        // records of the blocks' partial sums and, per matrix, the blocks that own a piece of it
-        std::vector<int> rec_off(spans.size() + 1, 0);
-        std::vector<BlockRange> owner(size_t(n), BlockRange{int(spans.size()), -1});
-        for (size_t k = 0; k < spans.size(); ++k) {
-            rec_off[k + 1] = rec_off[k] + (spans[k].z - spans[k].x + 1);
+        // per matrix: the blocks whose span holds it and where their records go
+        std::vector<DistOwner> owner(size_t(n), DistOwner{int(spans.size()), -1, 0});
+        for (size_t k = 0; k < spans.size(); ++k)
             for (int i = spans[k].x; i <= spans[k].z; ++i) {
-                owner[size_t(i)].x = std::min(owner[size_t(i)].x, int(k));
-                owner[size_t(i)].y = std::max(owner[size_t(i)].y, int(k));
+                owner[size_t(i)].first = std::min(owner[size_t(i)].first, int(k));
+                owner[size_t(i)].last = std::max(owner[size_t(i)].last, int(k));
             }
+        int n_rec = 0;
+        for (int i = 0; i < n; ++i) {
+            owner[size_t(i)].offset = n_rec;
+            n_rec += std::max(0, owner[size_t(i)].last - owner[size_t(i)].first + 1);
         }
-        if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_partial, sizeof(double) * 4 * size_t(std::max(1, rec_off.back())));
-        if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_rec_off, sizeof(int) * rec_off.size());
-        if (e == cudaSuccess) e = cudaMemcpy(b->d_dist_rec_off, rec_off.data(), sizeof(int) * rec_off.size(), cudaMemcpyHostToDevice);
-        if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_owner, sizeof(BlockRange) * size_t(n));
-        if (e == cudaSuccess) e = cudaMemcpy(b->d_dist_owner, owner.data(), sizeof(BlockRange) * size_t(n), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_partial, sizeof(double) * 4 * size_t(std::max(1, n_rec)));
+        if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_owner, sizeof(DistOwner) * size_t(n));
+        if (e == cudaSuccess) e = cudaMemcpy(b->d_dist_owner, owner.data(), sizeof(DistOwner) * size_t(n), cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = cudaMalloc(&b->d_dist_counter, sizeof(unsigned int));
         if (e == cudaSuccess) e = cudaMemset(b->d_dist_counter, 0, sizeof(unsigned int));
     }
@@ -1265,7 +1264,6 @@ extern "C" void qamw_batch_destroy(qamw_batch* b) {
     }
     if (b->d_spans_dist) cudaFree(b->d_spans_dist);
     if (b->d_dist_partial) cudaFree(b->d_dist_partial);
-    if (b->d_dist_rec_off) cudaFree(b->d_dist_rec_off);
     if (b->d_dist_owner) cudaFree(b->d_dist_owner);
     if (b->d_dist_counter) cudaFree(b->d_dist_counter);
     if (b->d_cal_all) cudaFree(b->d_cal_all);
@@ -1392,7 +1390,6 @@ extern "C" int qamw_distortion_batch(const qamw_batch* b, void* stream) {
     }
     DistReduce red;
     red.partial = b->d_dist_partial;
-    red.rec_off = b->d_dist_rec_off;
     red.owner = b->d_dist_owner;
     red.counter = b->d_dist_counter;
     return distortion_batch_launch(b->dec.d_descs, b->n, b->d_spans_dist, b->n_blocks_dist, b->w_dtype == QAMW_DTYPE_BF16,
