@@ -350,8 +350,15 @@ size_t qamw_batch_workspace_bytes(const qamw_batch* b);
 /* The four phases over all matrices of the batch, each equivalent to calling the single-matrix
  * entry point on every item in order (same results bit for bit, same error codes), asynchronous on
  * `stream`.  Matrices in the common layout (rows and metadata 16-byte aligned, d_in a multiple of
- * 16, block >= 32) are handled by one launch per phase; if any item falls outside, the phase falls
- * back to one launch per matrix. */
+ * 16, block >= 32) are handled by one launch per phase -- up to three in calibrate and encode, whose
+ * kernels run with one of three block sizes chosen by row length; if any item falls outside, the
+ * phase falls back to one launch per matrix.  Two exceptions to "bit for
+ * bit": the batched calibration groups the rows differently (pair scales agree to the last bits,
+ * about 1e-7 relative), and the batched distortion adds its partial sums in a fixed order, so its four
+ * sums are the same bits on every run (the single-matrix call uses atomic adds; both agree to about
+ * 1e-15 relative).  The handle owns a little device scratch for that (partial sums, a ticket
+ * counter that is zero between launches): calls on one batch must not overlap on the device, and a
+ * launch that was aborted leaves the distortion phase of that handle unusable (create a new one). */
 int qamw_calibrate_batch(const qamw_batch* b, void* workspace, size_t workspace_bytes, int32_t* status_out,
                          void* stream);
 int qamw_encode_batch(const qamw_batch* b, int32_t* status_out, void* stream);
