@@ -334,6 +334,7 @@ def run_ours(args):
         "quality": totals, "status_word": status_word, "wall_s_timed_region": t_wall,
     }
     out["fused_gemv"] = time_fused_gemv(mc, peak)
+    out["graph_step_ms"] = time_graph_step(mc, args.steps)
     if e2e is not None:
         out["e2e"] = e2e
     if e2e_full is not None:
@@ -357,6 +358,28 @@ def run_ours(args):
     print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_graph_step(mc, steps):
+    """The same step replayed as one CUDA graph (what a launch-bound small model should use); None if the
+    step cannot be captured."""
+    import torch
+
+    try:
+        graph = mc.capture_step()
+        for _ in range(3):
+            graph.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+    except Exception as exc:  # noqa: BLE001 - reported, not fatal: the eager timing above is the benchmark
+        sys.stderr.write(f"graph capture of the step failed: {exc}\n")
+        return None
 
 
 def time_fused_gemv(mc, peak_gbs, calls=50):

@@ -236,6 +236,20 @@ class ModelCodec:
         self.decode_all()
         self.distortion_all()
 
+    def capture_step(self) -> "torch.cuda.CUDAGraph":
+        """The whole step as one CUDA graph (seven kernel nodes and a memset for a batched model): replaying
+        it costs one launch, which is what small models need -- their kernels take a few microseconds
+        each and the per-call overhead of the host dominates otherwise.  The batched phases launch on the
+        current stream and allocate nothing, so they can be captured as they are."""
+        if not (self.use_batch and self.batch is not None):
+            raise RuntimeError("capture_step needs the batched phases (finalize() first)")
+        self.step()  # first use outside the capture: per-kernel attributes are set once
+        torch.cuda.synchronize(self.device)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.step()
+        return graph
+
     # --- accounting -----------------------------------------------------------------------------
     @property
     def n_weights(self) -> int:

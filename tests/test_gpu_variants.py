@@ -171,3 +171,24 @@ def test_fused_gemv_argument_errors():
     with pytest.raises(q.QamwError) as e:
         q.decode_gemv(dummy, f, None, dummy, f, cb, p, f[:192].reshape(3, 64), f[:12].reshape(4, 3), dummy)  # 3 vectors
     assert e.value.code == q.ERR_ARG
+
+
+def test_step_replayed_as_a_cuda_graph_gives_the_same_bytes():
+    """The batched step captured into one CUDA graph: replaying it reproduces the packed stream, the row
+    norms, the decoded matrices and the distortion sums of the eager step bit for bit."""
+    from paper_2605_26339_b200 import synth
+    from paper_2605_26339_b200.model_codec import ModelCodec
+    spec = synth.workload("cfg2", 256)
+    mc = ModelCodec.from_synthetic(spec, torch.device(DEV), load_golden_codebook(256), layers=[0])
+    mc.step()
+    torch.cuda.synchronize()
+    want = [(s.packed.clone(), s.row_norm.clone(), s.w_hat.clone(), s.dist.clone()) for s in mc.slots]
+    graph = mc.capture_step()
+    for s in mc.slots:
+        s.packed.zero_(); s.row_norm.zero_(); s.w_hat.zero_(); s.dist.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for s, (p, r, w, d) in zip(mc.slots, want):
+        assert torch.equal(s.packed, p) and torch.equal(s.row_norm, r)
+        assert torch.equal(s.w_hat.view(torch.int16), w.view(torch.int16)) and torch.equal(s.dist, d)
+    assert int(mc.status.cpu()[0]) == 0
