@@ -542,6 +542,17 @@ def test_polar_baseline_codec(orc, Ba, Bp, d_out, d_in, block, dtype):
     ref = orc.decode(enc["packed"], enc["row_norm"], block, cb.host, s, signs, sigma, d_in)
     ulps = np.abs(_bf16_ordered(_to_bits(what)) - _bf16_ordered(ref))
     assert (ulps <= 1).mean() > 1 - kFarFraction - 2.0 / ulps.size and (ulps == 0).mean() > 0.98
+    # the fused matrix-vector product works from the same reconstruction table
+    if d_in % 32 == 0:
+        g = torch.Generator().manual_seed(Ba + 3)
+        x = torch.randn((2, d_in), generator=g)
+        y = torch.full((d_out, 2), float("nan"), dtype=torch.float32, device=DEV)
+        q.decode_gemv(torch.from_numpy(enc["packed"]).to(DEV), torch.from_numpy(enc["row_norm"]).to(DEV), s_d, signs_d,
+                      sigma_d, cb, p, x.to(DEV), y)
+        _, w64 = orc.decode(enc["packed"], enc["row_norm"], block, cb.host, s, signs, sigma, d_in, want_f64=True)
+        x64 = x.numpy().astype(np.float64)
+        bound = 1e-5 * np.sqrt((w64 ** 2).sum(1))[:, None] * np.sqrt((x64 ** 2).sum(1))[None, :]
+        assert np.all(np.abs(y.cpu().numpy() - w64 @ x64.T) <= bound + 1e-30)
     print("PARITY polar", dict(Ba=Ba, Bp=Bp, pairs=int(idx.size), mismatches=int(diff.sum()), exempt=int(exempt.sum())))
 
 
