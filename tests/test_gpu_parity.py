@@ -629,3 +629,32 @@ def test_distortion_sums_for_short_and_ragged_streams(orc, d_out, d_in):
     batch.distortion()
     for d in dists:
         np.testing.assert_allclose(d.cpu().numpy(), ref, rtol=1e-9)
+
+
+def test_batch_with_the_polar_quantiser(orc):
+    """The batched phases take a polar codebook as they take a 2-D one: same bytes as the single-matrix
+    calls (whose indices test_polar_baseline_codec checks against the oracle)."""
+    Ba, Bp = 4, 4
+    shapes = [(130, 2048), (33, 11776), (64, 512)]
+    lv, _ = q.polar_train(Ba)
+    cb = q.Codebook.polar(lv, Ba, Bp)
+    _, a = _batch_problem(shapes, 256, 128, torch.bfloat16)
+    _, b = _batch_problem(shapes, 256, 128, torch.bfloat16)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for s in a:
+        ws = torch.empty(q.calibrate_workspace_bytes(s["p"]), dtype=torch.uint8, device=DEV)
+        q.calibrate(s["W"], s["p"], s["s"], s["signs"], s["sigma"], ws, st)
+        q.encode(s["W"], s["p"], s["s"], s["signs"], s["sigma"], cb, s["packed"], s["norm"], st)
+        q.decode(s["packed"], s["norm"], s["s"], s["signs"], s["sigma"], cb, s["p"], s["what"])
+    mats = [q.make_matrix(s["p"], s["W"], s["s"], s["signs"], s["sigma"], s["act"], s["packed"], s["norm"], s["what"],
+                          s["dist"]) for s in b]
+    batch = q.Batch(mats, cb)
+    for x, y in zip(a, b):
+        y["sigma"].copy_(x["sigma"])
+    batch.encode(st)
+    batch.decode()
+    torch.cuda.synchronize()
+    assert int(st.cpu()[0]) == 0
+    for x, y in zip(a, b):
+        assert torch.equal(x["packed"], y["packed"]) and torch.equal(x["norm"], y["norm"])
+        assert torch.equal(x["what"].view(torch.int16), y["what"].view(torch.int16))
